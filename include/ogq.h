@@ -1,0 +1,141 @@
+/*
+ * ogq.h -- C ABI of the optimal-gradient-quantization library (CUDA, sm_100a).
+ *
+ * The library implements the per-tensor quantization path of "Optimal Gradient
+ * Quantization Condition for Communication-Efficient Distributed Training":
+ * runtime level solvers for BinGrad-b, BinGrad-pb and ORQ, quantize + bit-pack,
+ * and the server-side unpack + dequantize + sum over K workers.
+ *
+ * Conventions shared by every entry point
+ *   - A bucket is a flat fp32 array `grad` of `total_elems` elements holding T
+ *     tensors back to back: tensor t is grad[off[t] .. off[t+1]), off[0] = 0,
+ *     off[T] = total_elems, off non-decreasing.  Empty tensors are allowed.
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; pointers named
+ *     h_* are HOST pointers.  d_grad, d_out and every packed buffer must be
+ *     16-byte aligned; tensor offsets need no alignment (tensors whose offset
+ *     is not a multiple of 4 elements take a scalar-load path).
+ *   - The library allocates no memory and keeps no state between calls.  Scratch
+ *     memory is the caller's `d_ws` of at least ogq_workspace_bytes(...) bytes,
+ *     256-byte aligned; its contents need not be preserved or initialised.
+ *   - Calls only enqueue work on `stream` and return at once.  The return code
+ *     reports argument validation and launch errors.  Conditions that depend on
+ *     the data are reported per tensor in d_status (bits OGQ_ST_*), never by a
+ *     trap.  There is no CPU fallback.
+ *   - Levels are fp32 because they are what a worker sends next to its codes.
+ */
+#ifndef OGQ_H_
+#define OGQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *ogq_stream_t; /* a cudaStream_t */
+
+typedef enum {
+    OGQ_OK = 0,
+    OGQ_ERR_INVALID_ARG = 1,
+    OGQ_ERR_UNSUPPORTED = 2,
+    OGQ_ERR_WORKSPACE = 3,
+    OGQ_ERR_CUDA = 4
+} ogq_status;
+
+typedef enum { OGQ_BINGRAD_PB = 0, OGQ_BINGRAD_B = 1, OGQ_ORQ = 2 } ogq_scheme;
+
+/* per-tensor status bits written to d_status */
+#define OGQ_ST_EMPTY 1      /* tensor has no elements; its levels are 0 */
+#define OGQ_ST_NONFINITE 2  /* NaN or Inf seen; levels are 0 (ORQ, pb) or unspecified (b) */
+#define OGQ_ST_CONSTANT 4   /* all elements equal (one side of the split empty): all levels equal */
+#define OGQ_ST_ITER_CAP 8   /* an iteration limit was reached before convergence */
+#define OGQ_ST_INTERNAL 16  /* a solver bracket failed to contain its target (should not happen) */
+
+/* Library version string (static storage). */
+const char *ogq_version(void);
+
+/* Code width in bits for s levels: 1 for s = 2, ceil(log2 s) otherwise; 0 if s < 2 or s > 32. */
+int ogq_bits_for_levels(int s);
+
+/*
+ * Packed layout (the paper's Algorithm 2 only says "encode"; this is the wire
+ * format of this library).  Per tensor a little-endian bit stream of 32-bit
+ * words: the code of element i occupies stream bits [i*bits, (i+1)*bits),
+ * stream bit j is bit (j mod 32) of word j/32, and each tensor's region is zero
+ * padded to a multiple of 4 words.  Fills h_packed_off[0..T] (in words) from
+ * the host copy of the element offsets.  Host-only; no device work.
+ */
+ogq_status ogq_packed_layout(const int64_t *h_off, int T, int bits, int64_t *h_packed_off);
+
+/*
+ * Upper bound of the scratch bytes any level solver needs for a bucket of
+ * `num_tensors` tensors and `total_elems` elements with at most `max_levels`
+ * levels.  Host-only.
+ */
+size_t ogq_workspace_bytes(int num_tensors, int64_t total_elems, int max_levels);
+
+/*
+ * BinGrad levels (Section "Binary Quantization").
+ *   variant OGQ_BINGRAD_B : Eq. (bingrad-b optimal condition).  b_0 starts at the
+ *     tensor mean; b_{-1}, b_1 are the means of {v < b_0} and {v >= b_0}.  With
+ *     lloyd_iters = I > 0 the update b_0 = (b_{-1} + b_1)/2 followed by new means
+ *     is applied up to I times, stopping when the split no longer changes
+ *     (OGQ_ST_ITER_CAP if it still changed after I updates).  b_0 is rounded to
+ *     fp32 at every step, since it is the threshold the quantizer compares with.
+ *   variant OGQ_BINGRAD_PB: Eq. (bingrad-pb optimal condition) on |v|: b_1 is where
+ *     g(b) = b n - sum_{|v| >= b} |v| changes sign (the minimiser of the
+ *     quantizer's squared error); levels are {-b_1, +b_1}; lloyd_iters is ignored.
+ * Outputs: d_levels [T][2] = {b_{-1}, b_1}; d_thresh [T] = b_0 (B only, may be
+ * NULL for PB); d_status [T].
+ */
+ogq_status ogq_levels_bingrad(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems,
+                              int variant, int lloyd_iters, float *d_levels, float *d_thresh,
+                              int32_t *d_status, void *d_ws, size_t ws_bytes, ogq_stream_t stream);
+
+/*
+ * ORQ levels (Algorithm 1 with the discrete form of the simplified optimal
+ * condition).  s in {3, 5, 9, 17}.  The end levels are the tensor's minimum and
+ * maximum (Corollary 1); every other level is the middle of its two bracket
+ * levels L < R: with T = sum_{L <= v <= R} (v - L) / (R - L), it is the
+ * (floor(T) + 1)-th largest element of {L <= v <= R}, so every level is one of
+ * the tensor's own values and the result is exact.
+ * Output: d_levels [T][s] ascending, d_status [T].
+ */
+ogq_status ogq_levels_orq(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems, int s,
+                          float *d_levels, int32_t *d_status, void *d_ws, size_t ws_bytes,
+                          ogq_stream_t stream);
+
+/*
+ * Quantize and pack (the random-rounding equation of Section "Multi-level
+ * Quantization", Eq. (bingrad-pb), Eq. (bingrad-b), then "encode").
+ *   ORQ / BINGRAD_PB (s = 2): segment k = 1 + #{interior levels <= v}, lo = b_{k-1},
+ *     hi = b_k; the code is k if  (float)u * (hi - lo) < (v - lo) * 2^24  (each
+ *     operation in fp32, round to nearest), else k - 1; u is the top 24 bits of
+ *     word (i mod 4) of Philox4x32-10 with key (seed low, seed high) and counter
+ *     (i/4 low, i/4 high, tensor index, stream_id), i the index inside the tensor.
+ *     Values outside [b_0, b_{s-1}] get the nearest end code.
+ *   BINGRAD_B: code = [v >= d_thresh[t]]; no random numbers; d_levels is unused.
+ * d_levels is [T][s], d_thresh is [T] (B only), d_packed_off [T+1] comes from
+ * ogq_packed_layout, d_packed receives d_packed_off[T] words (all of them are
+ * written, padding included).
+ */
+ogq_status ogq_quantize_pack(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems,
+                             ogq_scheme scheme, int s, const float *d_levels, const float *d_thresh,
+                             uint64_t seed, uint32_t stream_id, const int64_t *d_packed_off,
+                             uint32_t *d_packed, ogq_stream_t stream);
+
+/*
+ * Server step of Algorithm 2: out[i] = scale * sum_{k<K} levels_k[t][code_k[i]],
+ * summed in fp32 in worker order k = 0..K-1.  d_packed_k and d_levels_k are
+ * DEVICE arrays of K device pointers (worker k's packed buffer and its [T][s]
+ * level table).  1 <= K <= 64.  scale = 1/K gives the broadcast average.
+ */
+ogq_status ogq_unpack_sum(const uint32_t *const *d_packed_k, const float *const *d_levels_k, int K,
+                          const int64_t *d_off, const int64_t *d_packed_off, int T, int64_t total_elems,
+                          int s, float scale, float *d_out, ogq_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OGQ_H_ */

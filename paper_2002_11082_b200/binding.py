@@ -1,0 +1,151 @@
+"""ctypes binding of libogq.so: same names and argument order as include/ogq.h."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libogq.so")
+
+OGQ_BINGRAD_PB, OGQ_BINGRAD_B, OGQ_ORQ = 0, 1, 2
+OGQ_ST_EMPTY, OGQ_ST_NONFINITE, OGQ_ST_CONSTANT, OGQ_ST_ITER_CAP, OGQ_ST_INTERNAL = 1, 2, 4, 8, 16
+
+_STATUS_NAMES = {1: "OGQ_ERR_INVALID_ARG", 2: "OGQ_ERR_UNSUPPORTED", 3: "OGQ_ERR_WORKSPACE", 4: "OGQ_ERR_CUDA"}
+
+
+class OgqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where} failed: {_STATUS_NAMES.get(code, code)}")
+        self.code = code
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library.  Raises if libogq.so has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2002_11082_b200.build` "
+                "(nvcc, sm_100a); there is no CPU fallback"
+            )
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+        L.ogq_version.restype = ctypes.c_char_p
+        L.ogq_version.argtypes = []
+        L.ogq_bits_for_levels.restype = i32
+        L.ogq_bits_for_levels.argtypes = [i32]
+        L.ogq_packed_layout.restype = i32
+        L.ogq_packed_layout.argtypes = [vp, i32, i32, vp]
+        L.ogq_workspace_bytes.restype = sz
+        L.ogq_workspace_bytes.argtypes = [i32, i64, i32]
+        L.ogq_levels_bingrad.restype = i32
+        L.ogq_levels_bingrad.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.ogq_levels_orq.restype = i32
+        L.ogq_levels_orq.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, sz, vp]
+        L.ogq_quantize_pack.restype = i32
+        L.ogq_quantize_pack.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, ctypes.c_uint64, ctypes.c_uint32, vp, vp, vp]
+        L.ogq_unpack_sum.restype = i32
+        L.ogq_unpack_sum.argtypes = [vp, vp, i32, vp, vp, i32, i64, i32, ctypes.c_float, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Address of a torch tensor's storage, a raw integer address, or None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise OgqError(code, where)
+
+
+def ogq_version() -> str:
+    return lib().ogq_version().decode()
+
+
+def ogq_bits_for_levels(s: int) -> int:
+    return int(lib().ogq_bits_for_levels(int(s)))
+
+
+def ogq_packed_layout(h_off, bits: int) -> np.ndarray:
+    """Host helper: word offsets [T+1] of the packed regions for element offsets h_off [T+1]."""
+    h = np.ascontiguousarray(np.asarray(h_off), dtype=np.int64)
+    out = np.zeros_like(h)
+    _check(lib().ogq_packed_layout(h.ctypes.data, h.size - 1, int(bits), out.ctypes.data), "ogq_packed_layout")
+    return out
+
+
+def ogq_workspace_bytes(num_tensors: int, total_elems: int, max_levels: int) -> int:
+    return int(lib().ogq_workspace_bytes(int(num_tensors), int(total_elems), int(max_levels)))
+
+
+def ogq_levels_bingrad(d_grad, d_off, T: int, total_elems: int, variant: int, lloyd_iters: int,
+                       d_levels, d_thresh, d_status, d_ws, ws_bytes: int, stream=None) -> None:
+    _check(
+        lib().ogq_levels_bingrad(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(variant),
+                                 int(lloyd_iters), _ptr(d_levels), _ptr(d_thresh), _ptr(d_status),
+                                 _ptr(d_ws), int(ws_bytes), _stream(stream)),
+        "ogq_levels_bingrad",
+    )
+
+
+def ogq_levels_orq(d_grad, d_off, T: int, total_elems: int, s: int, d_levels, d_status, d_ws,
+                   ws_bytes: int, stream=None) -> None:
+    _check(
+        lib().ogq_levels_orq(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(s), _ptr(d_levels),
+                             _ptr(d_status), _ptr(d_ws), int(ws_bytes), _stream(stream)),
+        "ogq_levels_orq",
+    )
+
+
+def ogq_quantize_pack(d_grad, d_off, T: int, total_elems: int, scheme: int, s: int, d_levels, d_thresh,
+                      seed: int, stream_id: int, d_packed_off, d_packed, stream=None) -> None:
+    _check(
+        lib().ogq_quantize_pack(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(scheme), int(s),
+                                _ptr(d_levels), _ptr(d_thresh), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                int(stream_id) & 0xFFFFFFFF, _ptr(d_packed_off), _ptr(d_packed),
+                                _stream(stream)),
+        "ogq_quantize_pack",
+    )
+
+
+def ogq_unpack_sum(d_packed_k, d_levels_k, K: int, d_off, d_packed_off, T: int, total_elems: int, s: int,
+                   scale: float, d_out, stream=None) -> None:
+    _check(
+        lib().ogq_unpack_sum(_ptr(d_packed_k), _ptr(d_levels_k), int(K), _ptr(d_off), _ptr(d_packed_off),
+                             int(T), int(total_elems), int(s), float(scale), _ptr(d_out), _stream(stream)),
+        "ogq_unpack_sum",
+    )
+
+
+def device_pointer_array(tensors: Sequence, device=None):
+    """An int64 device tensor holding the data pointers of `tensors` (for ogq_unpack_sum)."""
+    import torch
+
+    dev = device if device is not None else tensors[0].device
+    return torch.tensor([t.data_ptr() for t in tensors], dtype=torch.int64, device=dev)

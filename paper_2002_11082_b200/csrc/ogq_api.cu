@@ -1,0 +1,146 @@
+// extern "C" entry points: argument validation, scratch layout, kernel launches.
+#include <cuda_runtime.h>
+
+#include "../../include/ogq.h"
+#include "ogq_internal.h"
+
+namespace {
+
+int sm_count_of_current_device()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return sms;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+bool valid_orq_levels(int s) { return s == 3 || s == 5 || s == 9 || s == 17; }
+
+}  // namespace
+
+extern "C" {
+
+const char* ogq_version(void) { return "ogq 0.1 (sm_100a)"; }
+
+int ogq_bits_for_levels(int s)
+{
+    if (s < 2 || s > 32) return 0;
+    int bits = 1;
+    while ((1 << bits) < s) ++bits;
+    return bits;
+}
+
+ogq_status ogq_packed_layout(const int64_t* h_off, int T, int bits, int64_t* h_packed_off)
+{
+    if (!h_off || !h_packed_off || T < 0 || bits < 1 || bits > 5) return OGQ_ERR_INVALID_ARG;
+    h_packed_off[0] = 0;
+    for (int t = 0; t < T; ++t) {
+        const int64_t n = h_off[t + 1] - h_off[t];
+        if (n < 0) return OGQ_ERR_INVALID_ARG;
+        const int64_t w = (n * bits + 31) / 32;
+        h_packed_off[t + 1] = h_packed_off[t] + (w + 3) / 4 * 4;
+    }
+    return OGQ_OK;
+}
+
+size_t ogq_workspace_bytes(int num_tensors, int64_t total_elems, int max_levels)
+{
+    if (num_tensors < 0 || total_elems < 0) return 0;
+    size_t a = ogq::ws_bytes_bingrad_b(num_tensors, total_elems);
+    size_t b = ogq::ws_bytes_select(num_tensors, total_elems, max_levels < 3 ? 3 : max_levels);
+    return (a > b ? a : b) + 256;
+}
+
+ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                              int variant, int lloyd_iters, float* d_levels, float* d_thresh,
+                              int32_t* d_status, void* d_ws, size_t ws_bytes, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_status || lloyd_iters < 0 ||
+        lloyd_iters > 1024)
+        return OGQ_ERR_INVALID_ARG;
+    if (variant != OGQ_BINGRAD_PB && variant != OGQ_BINGRAD_B) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
+    if (variant == OGQ_BINGRAD_B && !d_thresh) return OGQ_ERR_INVALID_ARG;
+    if (T == 0) return OGQ_OK;
+    if (!d_ws || ((uintptr_t)d_ws & 255u)) return OGQ_ERR_WORKSPACE;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e;
+    if (variant == OGQ_BINGRAD_B) {
+        if (ws_bytes < ogq::ws_bytes_bingrad_b(T, total_elems)) return OGQ_ERR_WORKSPACE;
+        e = ogq::launch_levels_bingrad_b(d_grad, d_off, T, total_elems, lloyd_iters, d_levels, d_thresh,
+                                         d_status, d_ws, sms, (cudaStream_t)stream);
+    } else {
+        if (ws_bytes < ogq::ws_bytes_select(T, total_elems, 2)) return OGQ_ERR_WORKSPACE;
+        e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_BINGRAD_PB, 2, d_levels, d_status,
+                                      d_ws, ws_bytes, sms, (cudaStream_t)stream);
+    }
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_levels_orq(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                          float* d_levels, int32_t* d_status, void* d_ws, size_t ws_bytes,
+                          ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_status) return OGQ_ERR_INVALID_ARG;
+    if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
+    if (T == 0) return OGQ_OK;
+    if (!d_ws || ((uintptr_t)d_ws & 255u)) return OGQ_ERR_WORKSPACE;
+    if (ws_bytes < ogq::ws_bytes_select(T, total_elems, s)) return OGQ_ERR_WORKSPACE;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_ORQ, s, d_levels, d_status,
+                                              d_ws, ws_bytes, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_quantize_pack(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                             ogq_scheme scheme, int s, const float* d_levels, const float* d_thresh,
+                             uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
+                             uint32_t* d_packed, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_packed_off) return OGQ_ERR_INVALID_ARG;
+    if (scheme == OGQ_BINGRAD_B) {
+        if (s != 2) return OGQ_ERR_UNSUPPORTED;
+        if (!d_thresh) return OGQ_ERR_INVALID_ARG;
+    } else if (scheme == OGQ_BINGRAD_PB) {
+        if (s != 2) return OGQ_ERR_UNSUPPORTED;
+        if (!d_levels) return OGQ_ERR_INVALID_ARG;
+    } else if (scheme == OGQ_ORQ) {
+        if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
+        if (!d_levels) return OGQ_ERR_INVALID_ARG;
+    } else {
+        return OGQ_ERR_UNSUPPORTED;
+    }
+    if (total_elems > 0 && (!d_grad || !d_packed || !aligned16(d_grad) || !aligned16(d_packed)))
+        return OGQ_ERR_INVALID_ARG;
+    if (T == 0 || total_elems == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_quantize_pack(d_grad, d_off, T, total_elems, (int)scheme, s, d_levels,
+                                              d_thresh, seed, stream_id, d_packed_off, d_packed, sms,
+                                              (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_unpack_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                          const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total_elems,
+                          int s, float scale, float* d_out, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_packed_off || !d_packed_k || !d_levels_k)
+        return OGQ_ERR_INVALID_ARG;
+    if (K < 1 || K > 64) return OGQ_ERR_INVALID_ARG;
+    if (!(s == 2 || valid_orq_levels(s))) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_out || !aligned16(d_out))) return OGQ_ERR_INVALID_ARG;
+    if (T == 0 || total_elems == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_unpack_sum(d_packed_k, d_levels_k, K, d_off, d_packed_off, T, total_elems, s,
+                                           scale, d_out, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+}  // extern "C"

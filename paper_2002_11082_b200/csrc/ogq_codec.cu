@@ -1,0 +1,241 @@
+// Quantize + bit-pack, and unpack + dequantize + sum over K workers.
+//
+// Both kernels walk the flat bucket in chunks.  Inside a tensor the unit of work
+// is a group of 128 consecutive elements (tensor-relative), which fills exactly
+// 4*bits output words; a group belongs to the CTA whose chunk holds its first
+// element, so no two CTAs ever touch the same word.  A warp takes one group per
+// iteration: lane l handles elements 4l..4l+3 (one 128-bit load, one Philox
+// block), and the words are assembled with shuffles inside each 8-lane set,
+// which produces exactly `bits` words.
+#include <math.h>
+
+#include "ogq_common.cuh"
+#include "ogq_internal.h"
+
+namespace ogq {
+
+constexpr int kMaxLevels = 32;
+constexpr int kMaxWorkers = 64;
+
+// OR-combine the 4*BITS-bit chunk of each lane into words; lane (8q + j), j < BITS,
+// returns word j of 8-lane set q.
+template <int BITS>
+__device__ __forceinline__ uint32_t assemble_words(uint32_t chunk, int lane)
+{
+    const int j = lane & 7;
+    const int bitpos = j * 4 * BITS;
+    const int w0 = bitpos >> 5, sh = bitpos & 31;
+    const uint32_t lo = chunk << sh;
+    const uint32_t hi = (sh + 4 * BITS > 32) ? (chunk >> (32 - sh)) : 0u;
+    uint32_t mine = 0;
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) {
+        uint32_t val = ((w0 == k) ? lo : 0u) | ((w0 + 1 == k) ? hi : 0u);
+        val |= __shfl_xor_sync(0xffffffffu, val, 1);
+        val |= __shfl_xor_sync(0xffffffffu, val, 2);
+        val |= __shfl_xor_sync(0xffffffffu, val, 4);
+        if (j == k) mine = val;
+    }
+    return mine;
+}
+
+template <int BITS, bool THRESHOLD>
+__global__ void __launch_bounds__(kThreads)
+k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off, int T, int64_t total,
+                int64_t chunk, int s, const float* __restrict__ levels, const float* __restrict__ thresh,
+                uint32_t seed_lo, uint32_t seed_hi, uint32_t stream_id,
+                const int64_t* __restrict__ packed_off, uint32_t* __restrict__ packed)
+{
+    __shared__ float sh_lv[kMaxLevels];
+    __shared__ float sh_w[kMaxLevels];
+
+    const int64_t lo = (int64_t)blockIdx.x * chunk;
+    const int64_t hi = (lo + chunk < total) ? lo + chunk : total;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    for_each_piece(off, T, lo, hi, [&](int t, int64_t tb, int64_t te, int64_t pb, int64_t pe) {
+        const int64_t n = te - tb;
+        const int64_t g_beg = (pb - tb + 127) >> 7, g_end = (pe - tb + 127) >> 7;
+        if (g_beg >= g_end) return;
+        float b0 = 0.f;
+        if (THRESHOLD) {
+            b0 = __ldg(thresh + t);
+        } else {
+            __syncthreads();
+            if (threadIdx.x < s) {
+                const float cur = __ldg(levels + (int64_t)t * s + threadIdx.x);
+                const float prv = threadIdx.x > 0 ? __ldg(levels + (int64_t)t * s + threadIdx.x - 1) : cur;
+                sh_lv[threadIdx.x] = cur;
+                sh_w[threadIdx.x] = __fsub_rn(cur, prv);  // width of the segment below level k
+            }
+            __syncthreads();
+        }
+        const int64_t region = __ldg(packed_off + t + 1) - __ldg(packed_off + t);
+        uint32_t* out = packed + __ldg(packed_off + t);
+        const bool aligned = (tb & 3) == 0;
+        const float* base = grad + tb;
+
+        for (int64_t g = g_beg + warp; g < g_end; g += kWarps) {
+            const int64_t i0 = (g << 7) + 4 * lane;
+            float x[4];
+            if (aligned && i0 + 3 < n) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(base + i0));
+                x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) x[j] = (i0 + j < n) ? __ldg(base + i0 + j) : 0.f;
+            }
+            uint32_t c[4];
+            if (THRESHOLD) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) c[j] = (x[j] >= b0) ? 1u : 0u;
+            } else {
+                const uint64_t q = (uint64_t)i0 >> 2;
+                const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)t, stream_id,
+                                              seed_lo, seed_hi);
+                const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    int idx = 0;
+                    for (int step = (s - 1) >> 1; step >= 1; step >>= 1)
+                        if (sh_lv[idx + step] <= x[j]) idx += step;
+                    const float d = __fsub_rn(x[j], sh_lv[idx]);
+                    const float lhs = __fmul_rn((float)(rw[j] >> 8), sh_w[idx + 1]);
+                    const float rhs = __fmul_rn(d, 16777216.0f);
+                    c[j] = (uint32_t)idx + ((lhs < rhs) ? 1u : 0u);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j >= n) c[j] = 0u;  // zero padding beyond the tensor
+            const uint32_t bits4 = c[0] | (c[1] << BITS) | (c[2] << (2 * BITS)) | (c[3] << (3 * BITS));
+            const uint32_t word = assemble_words<BITS>(bits4, lane);
+            const int j8 = lane & 7;
+            if (j8 < BITS) {
+                const int64_t widx = g * (4 * BITS) + (lane >> 3) * BITS + j8;
+                if (widx < region) out[widx] = word;
+            }
+        }
+    });
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kThreads)
+k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* __restrict__ levels_k, int K,
+             const int64_t* __restrict__ off, const int64_t* __restrict__ packed_off, int T, int64_t total,
+             int64_t chunk, int s, float scale, float* __restrict__ outp)
+{
+    __shared__ float sh_lv[kMaxWorkers][kMaxLevels + 1];
+    __shared__ const uint32_t* sh_pk[kMaxWorkers];
+
+    const int64_t lo = (int64_t)blockIdx.x * chunk;
+    const int64_t hi = (lo + chunk < total) ? lo + chunk : total;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr uint32_t kMask4 = (BITS * 4 >= 32) ? 0xffffffffu : ((1u << (BITS * 4)) - 1u);
+    constexpr uint32_t kMask1 = (1u << BITS) - 1u;
+
+    for_each_piece(off, T, lo, hi, [&](int t, int64_t tb, int64_t te, int64_t pb, int64_t pe) {
+        const int64_t n = te - tb;
+        const int64_t g_beg = (pb - tb + 127) >> 7, g_end = (pe - tb + 127) >> 7;
+        if (g_beg >= g_end) return;
+        __syncthreads();
+        for (int i = threadIdx.x; i < K * s; i += kThreads) {
+            const int k = i / s, q = i - k * s;
+            sh_lv[k][q] = __ldg(levels_k[k] + (int64_t)t * s + q);
+        }
+        const int64_t pofs = __ldg(packed_off + t);
+        if (threadIdx.x < K) sh_pk[threadIdx.x] = packed_k[threadIdx.x] + pofs;
+        __syncthreads();
+        const int64_t region = __ldg(packed_off + t + 1) - pofs;
+        const bool aligned = (tb & 3) == 0;
+        float* dst = outp + tb;
+
+        for (int64_t g = g_beg + warp; g < g_end; g += kWarps) {
+            const int64_t i0 = (g << 7) + 4 * lane;
+            if (i0 >= n) continue;
+            const int64_t bit = i0 * BITS;
+            const int64_t wi = bit >> 5;
+            const int sh = (int)(bit & 31);
+            const bool two = (sh + 4 * BITS > 32) && (wi + 1 < region);
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int k = 0; k < K; ++k) {
+                const uint32_t* p = sh_pk[k];
+                const uint32_t w_lo = __ldg(p + wi);
+                const uint32_t w_hi = two ? __ldg(p + wi + 1) : 0u;
+                const uint32_t bits4 = __funnelshift_r(w_lo, w_hi, sh) & kMask4;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t code = (bits4 >> (j * BITS)) & kMask1;
+                    if (code > (uint32_t)(s - 1)) code = (uint32_t)(s - 1);
+                    acc[j] = __fadd_rn(acc[j], sh_lv[k][code]);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] = __fmul_rn(acc[j], scale);
+            if (aligned && i0 + 3 < n) {
+                *reinterpret_cast<float4*>(dst + i0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j < n) dst[i0 + j] = acc[j];
+            }
+        }
+    });
+}
+
+static int flat_target(int sm_count)
+{
+    int t = sm_count * 8;
+    return t < kMaxFlatCtas ? t : kMaxFlatCtas;
+}
+
+cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int T, int64_t total,
+                                 int scheme, int s, const float* d_levels, const float* d_thresh,
+                                 uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
+                                 uint32_t* d_packed, int sm_count, cudaStream_t stream)
+{
+    FlatGrid g = make_flat_grid(total, flat_target(sm_count), 8192);
+    const uint32_t slo = (uint32_t)seed, shi = (uint32_t)(seed >> 32);
+    const int bits = ogq_bits_for_levels(s);
+#define OGQ_LAUNCH_Q(B, TH)                                                                          \
+    k_quantize_pack<B, TH><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, s,     \
+                                                            d_levels, d_thresh, slo, shi, stream_id, \
+                                                            d_packed_off, d_packed)
+    if (scheme == OGQ_BINGRAD_B) {
+        OGQ_LAUNCH_Q(1, true);
+    } else {
+        switch (bits) {
+            case 1: OGQ_LAUNCH_Q(1, false); break;
+            case 2: OGQ_LAUNCH_Q(2, false); break;
+            case 3: OGQ_LAUNCH_Q(3, false); break;
+            case 4: OGQ_LAUNCH_Q(4, false); break;
+            case 5: OGQ_LAUNCH_Q(5, false); break;
+            default: return cudaErrorInvalidValue;
+        }
+    }
+#undef OGQ_LAUNCH_Q
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                              const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total,
+                              int s, float scale, float* d_out, int sm_count, cudaStream_t stream)
+{
+    FlatGrid g = make_flat_grid(total, flat_target(sm_count), 8192);
+    const int bits = ogq_bits_for_levels(s);
+#define OGQ_LAUNCH_U(B)                                                                               \
+    k_unpack_sum<B><<<g.ctas, kThreads, 0, stream>>>(d_packed_k, d_levels_k, K, d_off, d_packed_off, T, \
+                                                     total, g.chunk, s, scale, d_out)
+    switch (bits) {
+        case 1: OGQ_LAUNCH_U(1); break;
+        case 2: OGQ_LAUNCH_U(2); break;
+        case 3: OGQ_LAUNCH_U(3); break;
+        case 4: OGQ_LAUNCH_U(4); break;
+        case 5: OGQ_LAUNCH_U(5); break;
+        default: return cudaErrorInvalidValue;
+    }
+#undef OGQ_LAUNCH_U
+    return cudaGetLastError();
+}
+
+}  // namespace ogq

@@ -1,0 +1,170 @@
+// Shared device helpers of the gradient-quantization kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ogq.h"
+
+namespace ogq {
+
+constexpr int kThreads = 256;       // threads per CTA of every streaming kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kChunkAlign = 1024;   // flat chunk boundaries are multiples of this many elements
+
+// ---------------------------------------------------------------------------
+// Flat partition of the bucket: CTA c owns elements [c*chunk, (c+1)*chunk).
+// ---------------------------------------------------------------------------
+struct FlatGrid {
+    int64_t chunk;  // elements per CTA, multiple of kChunkAlign
+    int ctas;       // number of CTAs
+};
+
+inline FlatGrid make_flat_grid(int64_t total, int target_ctas, int64_t min_chunk)
+{
+    FlatGrid g;
+    if (total <= 0) {
+        g.chunk = kChunkAlign;
+        g.ctas = 1;
+        return g;
+    }
+    int64_t c = (total + target_ctas - 1) / target_ctas;
+    if (c < min_chunk) c = min_chunk;
+    c = (c + kChunkAlign - 1) / kChunkAlign * kChunkAlign;
+    g.chunk = c;
+    g.ctas = (int)((total + c - 1) / c);
+    return g;
+}
+
+// Largest t < T with off[t] <= x (the tensor that contains flat index x).
+__device__ __forceinline__ int find_tensor(const int64_t* __restrict__ off, int T, int64_t x)
+{
+    int lo = 0, hi = T;  // answer in [lo, hi)
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(off + mid) <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Calls f(t, tensor_begin, tensor_end, piece_begin, piece_end) for every non-empty
+// intersection of the flat range [lo, hi) with a tensor, in ascending order.
+template <class F>
+__device__ __forceinline__ void for_each_piece(const int64_t* __restrict__ off, int T, int64_t lo,
+                                               int64_t hi, F f)
+{
+    if (lo >= hi || T <= 0) return;
+    int t = find_tensor(off, T, lo);
+    int64_t pos = lo;
+    while (pos < hi && t < T) {
+        int64_t tb = __ldg(off + t), te = __ldg(off + t + 1);
+        int64_t pe = te < hi ? te : hi;
+        if (pe > pos) {
+            f(t, tb, te, pos, pe);
+            pos = pe;
+        }
+        if (pe >= te) ++t;
+    }
+}
+
+// Block-cooperative visit of grad[pb, pe): 128-bit loads on the aligned body,
+// scalar loads on the ragged head and tail.  f(float) is called once per element.
+template <class F>
+__device__ __forceinline__ void visit_piece(const float* __restrict__ grad, int64_t pb, int64_t pe, F f)
+{
+    int64_t a = (pb + 3) & ~(int64_t)3;
+    if (a > pe) a = pe;
+    int64_t b = pe & ~(int64_t)3;
+    if (b < a) b = a;
+    const int tid = threadIdx.x;
+    if (tid < (int)(a - pb)) f(__ldg(grad + pb + tid));
+    if (tid < (int)(pe - b)) f(__ldg(grad + b + tid));
+    const float4* g4 = reinterpret_cast<const float4*>(grad);
+    int64_t i = (a >> 2) + tid, e = b >> 2;
+    for (; i + 3 * kThreads < e; i += 4 * kThreads) {
+        float4 x0 = __ldg(g4 + i);
+        float4 x1 = __ldg(g4 + i + kThreads);
+        float4 x2 = __ldg(g4 + i + 2 * kThreads);
+        float4 x3 = __ldg(g4 + i + 3 * kThreads);
+        f(x0.x); f(x0.y); f(x0.z); f(x0.w);
+        f(x1.x); f(x1.y); f(x1.z); f(x1.w);
+        f(x2.x); f(x2.y); f(x2.z); f(x2.w);
+        f(x3.x); f(x3.y); f(x3.z); f(x3.w);
+    }
+    for (; i < e; i += kThreads) {
+        float4 x = __ldg(g4 + i);
+        f(x.x); f(x.y); f(x.z); f(x.w);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Order-preserving map between fp32 values and unsigned 32-bit keys.
+// -0.0 is folded onto +0.0 first so that equal values have equal keys.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t float_to_key(float v)
+{
+    uint32_t b = __float_as_uint(v);
+    if (b == 0x80000000u) b = 0u;
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ float key_to_float(uint32_t k)
+{
+    uint32_t b = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+    return __uint_as_float(b);
+}
+
+// ---------------------------------------------------------------------------
+// Philox4x32 with 10 rounds (Salmon et al., SC'11).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+        uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = h1 ^ c1 ^ k0;
+        uint32_t n2 = h0 ^ c3 ^ k1;
+        c0 = n0; c1 = l1; c2 = n2; c3 = l0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// ---------------------------------------------------------------------------
+// Warp / block reductions with a fixed combination order (reproducible).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ long long warp_sum(long long x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Sum over the CTA; the result is valid in thread 0.  `scratch` holds kWarps values.
+template <class Tv>
+__device__ __forceinline__ Tv block_sum(Tv x, Tv* scratch)
+{
+    x = warp_sum(x);
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+    __syncthreads();
+    if (l == 0) scratch[w] = x;
+    __syncthreads();
+    Tv r = 0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) r += scratch[i];
+    }
+    return r;
+}
+
+}  // namespace ogq

@@ -1,0 +1,31 @@
+// Host-side launchers behind the C ABI (one per kernel family).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace ogq {
+
+constexpr int kMaxFlatCtas = 4096;  // upper bound on CTAs of a flat streaming grid (scratch sizing)
+
+cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, int T, int64_t total,
+                                    int lloyd_iters, float* d_levels, float* d_thresh, int32_t* d_status,
+                                    void* d_ws, int sm_count, cudaStream_t stream);
+size_t ws_bytes_bingrad_b(int T, int64_t total);
+
+cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int T, int64_t total,
+                                 int scheme, int s, float* d_levels, int32_t* d_status, void* d_ws,
+                                 size_t ws_bytes, int sm_count, cudaStream_t stream);
+size_t ws_bytes_select(int T, int64_t total, int s);
+
+cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int T, int64_t total,
+                                 int scheme, int s, const float* d_levels, const float* d_thresh,
+                                 uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
+                                 uint32_t* d_packed, int sm_count, cudaStream_t stream);
+
+cudaError_t launch_unpack_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                              const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total,
+                              int s, float scale, float* d_out, int sm_count, cudaStream_t stream);
+
+}  // namespace ogq

@@ -1,0 +1,1189 @@
+// ORQ and BinGrad-pb level solvers: exact selection by histogram refinement.
+//
+// Round 1 streams the bucket once: per tensor it finds min, max and a histogram
+// over key cells (128 cells per binade inside a 16-binade window anchored at a
+// sampled magnitude, one cell per binade outside), each cell with an exact
+// count and an exact integer sum of the low key bits.  The last CTA to finish a
+// tensor runs the scalar solver (ogq_select_solver.cuh), which turns the cell
+// prefix sums into a few narrow candidate intervals.  Round 2 streams the bucket
+// again, copies the few percent of elements inside the intervals to scratch and
+// histograms them on a finer grid; round 3 and later work on the copied keys
+// only, until every level's rank falls into a single-key cell.  Tensors of at
+// most kSmallN elements are sorted in shared memory instead.
+//
+// All cross-CTA accumulation is integer (atomic adds, min, max), and the
+// per-tensor prefix sums are built in a fixed order, so results are
+// bit-reproducible.  No kernel waits on another CTA: the "last CTA to arrive"
+// is found with one atomic counter per tensor.
+#include <math.h>
+
+#include "ogq_common.cuh"
+#include "ogq_internal.h"
+#include "ogq_select_solver.cuh"
+#include "ogq_ws.h"
+
+namespace ogq {
+
+constexpr int kSelW = 16;          // binades in the fine window of round 1
+constexpr int kSelM = 7;           // log2(cells per binade) in the window
+constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
+constexpr int kStageCap = 512;     // per-warp staging entries for compaction
+constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
+constexpr int kSliceElems = 16384;
+constexpr int kMaxRounds = 32;
+constexpr int kSortScanMax = 65536;  // longest copied-key list one CTA filters for the sorting finish
+
+static_assert(2 * (256 - kSelW + (kSelW << kSelM)) <= kCells, "round-1 cells exceed the budget");
+
+struct TState {
+    int done, round, m, status;
+    unsigned kmin_inv, kmax, nonfinite, arrive;
+    unsigned expected, pad0;
+    unsigned long long cursor[2];
+    long long n;
+    double stot;
+    Interval iv[kMaxIv];
+    ExactLv lv[kMaxLv];
+};
+
+struct SelWs {
+    TState* st;                  // [T]
+    uint32_t* gcnt;              // [T][kCells]
+    unsigned long long* glsum;   // [T][kCells]
+    unsigned* nitems;            // [1] work items of round 3
+    int2* items;                 // [T * kMaxSlices]
+    uint32_t* buf[2];            // [total] copied keys, tensor t at its element offset
+};
+
+static size_t sel_zero_bytes(int T)
+{
+    return align_up(sizeof(TState) * (size_t)T, 256) + align_up(sizeof(uint32_t) * (size_t)T * kCells, 256) +
+           align_up(sizeof(unsigned long long) * (size_t)T * kCells, 256) + 256;
+}
+
+size_t ws_bytes_select(int T, int64_t total, int /*s*/)
+{
+    return sel_zero_bytes(T) + align_up(sizeof(int2) * (size_t)T * kMaxSlices, 256) +
+           2 * align_up(sizeof(uint32_t) * (size_t)(total + 4), 256);
+}
+
+static SelWs sel_carve(void* base, int T, int64_t total)
+{
+    char* p = (char*)base;
+    SelWs w;
+    w.st = (TState*)p; p += align_up(sizeof(TState) * (size_t)T, 256);
+    w.gcnt = (uint32_t*)p; p += align_up(sizeof(uint32_t) * (size_t)T * kCells, 256);
+    w.glsum = (unsigned long long*)p; p += align_up(sizeof(unsigned long long) * (size_t)T * kCells, 256);
+    w.nitems = (unsigned*)p; p += 256;
+    w.items = (int2*)p; p += align_up(sizeof(int2) * (size_t)T * kMaxSlices, 256);
+    w.buf[0] = (uint32_t*)p; p += align_up(sizeof(uint32_t) * (size_t)(total + 4), 256);
+    w.buf[1] = (uint32_t*)p;
+    return w;
+}
+
+// ---------------------------------------------------------------------------
+// Shared-memory layout of a streaming CTA (dynamic): cell counters, low-bit sums
+// (two 32-bit halves with carry), and the per-warp compaction stages.  The
+// solver reuses the same bytes for its prefix arrays.
+// ---------------------------------------------------------------------------
+constexpr size_t kSmemHist = 3 * kCells * sizeof(uint32_t);
+constexpr size_t kSmemStage = kWarps * kStageCap * sizeof(uint32_t);
+constexpr size_t kSmemSolver = kSlots * (sizeof(uint32_t) + sizeof(double)) + 16;
+constexpr size_t kSmemBytes = (kSmemHist + kSmemStage > kSmemSolver) ? kSmemHist + kSmemStage : kSmemSolver;
+
+struct Table {  // interval lookup table of the tensor being streamed
+    uint32_t klo[kMaxIv];
+    uint32_t khi[kMaxIv];
+    int sh[kMaxIv];
+    int cellbase[kMaxIv];
+    int m, ncells;
+};
+
+__device__ __forceinline__ void table_from_intervals(Table& tb, const Interval* iv, int m)
+{
+    // called by one thread
+    int nc = 0;
+    for (int j = 0; j < kMaxIv; ++j) {
+        if (j < m) {
+            tb.klo[j] = iv[j].klo; tb.khi[j] = iv[j].khi; tb.sh[j] = iv[j].sh; tb.cellbase[j] = iv[j].cellbase;
+            nc = iv[j].cellbase + iv[j].ncell;
+        } else {
+            tb.klo[j] = 0xffffffffu; tb.khi[j] = 0u; tb.sh[j] = 0; tb.cellbase[j] = 0;
+        }
+    }
+    tb.m = m;
+    tb.ncells = nc;
+}
+
+// Round-1 intervals: coarse (one cell per binade) outside a window of kSelW binades that ends
+// at binade hi_e, fine inside.  Negative values only for signed keys.
+__device__ __forceinline__ int round1_intervals(int hi_e, bool magnitude_only, Interval* iv)
+{
+    const int lo_e = hi_e - kSelW;
+    int m = 0, cb = 0;
+    auto add = [&](uint32_t klo, int ncell, int sh) {
+        if (ncell <= 0) return;
+        Interval& x = iv[m++];
+        x.klo = klo; x.sh = sh; x.ncell = ncell;
+        x.khi = klo + (uint32_t)((((unsigned long long)ncell) << sh) - 1ull);
+        x.cellbase = cb; x.pad = 0; x.cbefore = 0; x.sbefore = 0.0;
+        cb += ncell;
+    };
+    if (!magnitude_only) {
+        add(0u, 256 - hi_e, 23);
+        add(0x80000000u - ((uint32_t)hi_e << 23), kSelW << kSelM, 23 - kSelM);
+        add(0x80000000u - ((uint32_t)lo_e << 23), lo_e, 23);
+    }
+    add(0x80000000u, lo_e, 23);
+    add(0x80000000u + ((uint32_t)lo_e << 23), kSelW << kSelM, 23 - kSelM);
+    add(0x80000000u + ((uint32_t)hi_e << 23), 256 - hi_e, 23);
+    return m;
+}
+
+__device__ __forceinline__ bool classify(const Table& tb, uint32_t key, int& cell, uint32_t& low, int& sh)
+{
+    int idx = 0;
+#pragma unroll
+    for (int step = kMaxIv / 2; step >= 1; step >>= 1)
+        if (tb.klo[idx + step] <= key) idx += step;
+    sh = tb.sh[idx];
+    const uint32_t rel = key - tb.klo[idx];
+    cell = tb.cellbase[idx] + (int)(rel >> sh);
+    low = rel & ((1u << sh) - 1u);
+    return key >= tb.klo[idx] && key <= tb.khi[idx];
+}
+
+__device__ __forceinline__ void hist_add(uint32_t* cnt, uint32_t* lo, uint32_t* hi, int cell, uint32_t low)
+{
+    atomicAdd(cnt + cell, 1u);
+    if (low) {
+        const uint32_t old = atomicAdd(lo + cell, low);
+        if (old + low < old) atomicAdd(hi + cell, 1u);
+    }
+}
+
+// Warp-uniform visit of base[pb, pe): every lane of a warp calls f(x, nvalid) the same number of
+// times (nvalid = 0, 1 or 4), so f may use warp collectives.  128-bit loads on the aligned body.
+__device__ __forceinline__ float4 ld4(const float4* p) { return __ldg(p); }
+__device__ __forceinline__ uint4 ld4(const uint4* p) { return __ldcg(p); }
+__device__ __forceinline__ float ld1(const float* p) { return __ldg(p); }
+__device__ __forceinline__ uint32_t ld1(const uint32_t* p) { return __ldcg(p); }
+
+template <class E4, class E, class F>
+__device__ __forceinline__ void warp_visit4(const E* __restrict__ base, int64_t pb, int64_t pe, F f)
+{
+    int64_t a = (pb + 3) & ~(int64_t)3;
+    if (a > pe) a = pe;
+    int64_t b = pe & ~(int64_t)3;
+    if (b < a) b = a;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (warp == 0) {
+        E x[4];
+        int nv = 0;
+        if (lane < (int)(a - pb)) { x[0] = ld1(base + pb + lane); nv = 1; }
+        else if (lane >= 4 && lane - 4 < (int)(pe - b)) { x[0] = ld1(base + b + lane - 4); nv = 1; }
+        f(x, nv);
+    }
+    const E4* b4 = reinterpret_cast<const E4*>(base);
+    const int64_t e = b >> 2;
+    for (int64_t i0 = (a >> 2) + warp * 32; i0 < e; i0 += 2 * kThreads) {
+        const int64_t i = i0 + lane, i2 = i + kThreads;
+        E x[4], y[4];
+        int nx = 0, ny = 0;
+        if (i < e) { const E4 v = ld4(b4 + i); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; nx = 4; }
+        if (i2 < e) { const E4 v = ld4(b4 + i2); y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w; ny = 4; }
+        f(x, nx);
+        if (i0 + kThreads < e) f(y, ny);
+    }
+}
+
+struct Stager {  // per-warp compaction stage
+    uint32_t* stage;            // this warp's kStageCap entries in shared memory
+    uint32_t* dst;              // tensor's region in the destination buffer
+    unsigned long long* cursor; // tensor's append cursor
+    int fill;
+
+    __device__ __forceinline__ void flush()
+    {
+        const int lane = threadIdx.x & 31;
+        if (fill > 0) {
+            unsigned long long pos = 0;
+            if (lane == 0) pos = atomicAdd(cursor, (unsigned long long)fill);
+            pos = __shfl_sync(0xffffffffu, pos, 0);
+            for (int i = lane; i < fill; i += 32) dst[pos + i] = stage[i];
+        }
+        __syncwarp();
+        fill = 0;
+    }
+
+    // every lane passes its own keys (c of them, c <= 4)
+    __device__ __forceinline__ void append(const uint32_t* kk, int c)
+    {
+        const int lane = threadIdx.x & 31;
+        int incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += nb;
+        }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        if (total == 0) return;
+        const int at = fill + incl - c;
+        for (int i = 0; i < c; ++i) stage[at + i] = kk[i];
+        fill += total;
+        __syncwarp();
+        if (fill > kStageCap - 128) flush();
+    }
+};
+
+// Streams one piece of a tensor's working set: histogram of the keys inside the intervals,
+// optional copy of those keys, and (round 1) min / max / non-finite tracking.
+template <bool FIRST, bool FROM_GRAD, bool COMPACT>
+__device__ __forceinline__ void stream_piece(const void* __restrict__ src, int64_t pb, int64_t pe,
+                                             bool magnitude_only, const Table& tb, uint32_t* cnt,
+                                             uint32_t* lo, uint32_t* hi, Stager& stg, uint32_t& kmin,
+                                             uint32_t& kmax, uint32_t& nonfinite)
+{
+    auto handle = [&](uint32_t key, uint32_t* kk, int& c) {
+        int cell, sh;
+        uint32_t low;
+        if (classify(tb, key, cell, low, sh)) {
+            hist_add(cnt, lo, hi, cell, low);
+            if (COMPACT) kk[c++] = key;
+        }
+    };
+    if (FROM_GRAD) {
+        warp_visit4<float4, float>((const float*)src, pb, pe, [&](const float* x, int nv) {
+            uint32_t kk[4];
+            int c = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (j < nv) {
+                    uint32_t bits = __float_as_uint(x[j]);
+                    if (FIRST && (bits & 0x7f800000u) == 0x7f800000u) nonfinite = 1u;
+                    uint32_t key;
+                    if (magnitude_only) key = bits | 0x80000000u;
+                    else {
+                        if (bits == 0x80000000u) bits = 0u;
+                        key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+                    }
+                    if (FIRST) { kmin = key < kmin ? key : kmin; kmax = key > kmax ? key : kmax; }
+                    handle(key, kk, c);
+                }
+            }
+            if (COMPACT) stg.append(kk, c);
+        });
+    } else {
+        warp_visit4<uint4, uint32_t>((const uint32_t*)src, pb, pe, [&](const uint32_t* x, int nv) {
+            uint32_t kk[4];
+            int c = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < nv) handle(x[j], kk, c);
+            if (COMPACT) stg.append(kk, c);
+        });
+    }
+}
+
+__device__ __forceinline__ void zero_hist(uint32_t* smem_hist, int ncells)
+{
+    for (int i = threadIdx.x; i < ncells; i += kThreads) {
+        smem_hist[i] = 0u;
+        smem_hist[kCells + i] = 0u;
+        smem_hist[2 * kCells + i] = 0u;
+    }
+}
+
+__device__ __forceinline__ void flush_hist(const uint32_t* smem_hist, int ncells, uint32_t* gcnt,
+                                           unsigned long long* glsum)
+{
+    for (int i = threadIdx.x; i < ncells; i += kThreads) {
+        const uint32_t c = smem_hist[i];
+        if (c) {
+            atomicAdd(gcnt + i, c);
+            const unsigned long long l =
+                ((unsigned long long)smem_hist[2 * kCells + i] << 32) | smem_hist[kCells + i];
+            if (l) atomicAdd(glsum + i, l);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Block-wide exclusive scan of (count, sum) pairs in thread order (fixed order).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void block_excl_scan(unsigned long long& c, double& s, unsigned long long* sc,
+                                                double* ss, unsigned long long& tot_c, double& tot_s)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long ic = c;
+    double is = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long nc = __shfl_up_sync(0xffffffffu, ic, o);
+        const double ns = __shfl_up_sync(0xffffffffu, is, o);
+        if (lane >= o) { ic += nc; is = ns + is; }
+    }
+    const unsigned long long pc = __shfl_up_sync(0xffffffffu, ic, 1);
+    const double ps = __shfl_up_sync(0xffffffffu, is, 1);
+    __syncthreads();
+    if (lane == 31) { sc[warp] = ic; ss[warp] = is; }
+    __syncthreads();
+    unsigned long long bc = 0;
+    double bs = 0.0;
+    tot_c = 0;
+    tot_s = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        if (w < warp) { bc += sc[w]; bs += ss[w]; }
+        tot_c += sc[w];
+        tot_s += ss[w];
+    }
+    c = (lane == 0) ? bc : bc + pc;
+    s = (lane == 0) ? bs : bs + ps;
+}
+
+struct SolverShared {
+    Interval iv[kMaxIv];
+    Interval niv[kMaxIv];
+    LvInfo lv[kMaxLv];
+    SolverView view;
+    unsigned long long sc[kWarps];
+    double ss[kWarps];
+    int pb_a, pb_b, pb_c;
+    int done, nm, internal;
+    long long cand;           // elements inside the new intervals
+    int n_keys, n_unique;     // sorting finish
+    int ivstart[kMaxIv], ivufirst[kMaxIv];
+    double ivpre[kMaxIv];
+};
+
+__device__ __forceinline__ int find_new_interval(const SolverShared& S, uint32_t key)
+{
+    int lo = 0, hi = S.nm;  // last interval with klo <= key
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (S.niv[mid].klo <= key) lo = mid; else hi = mid;
+    }
+    return (key >= S.niv[lo].klo && key <= S.niv[lo].khi) ? lo : -1;
+}
+
+// Sorting finish (ORQ): when the elements left inside the candidate intervals fit in shared
+// memory, they are sorted, run-length encoded into single-key cells with exact prefix counts
+// and sums, and one more solver pass resolves every open level at once.
+__device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long long src_cnt,
+                            float* __restrict__ levels, int32_t* __restrict__ status, unsigned char* smem,
+                            SolverShared& S)
+{
+    constexpr int kPer = kSmallN / kThreads;
+    uint32_t* skeys = reinterpret_cast<uint32_t*>(smem);
+    uint32_t* xkeys = skeys + kSmallN;
+    uint32_t* xcpre = xkeys + kSmallN;
+    double* xspre = reinterpret_cast<double*>(smem + ((3 * kSmallN + kMaxIv + 2) * sizeof(uint32_t) + 15) / 16 * 16);
+    __syncthreads();
+    if (threadIdx.x == 0) S.n_keys = 0;
+    if (threadIdx.x < kMaxIv) { S.ivstart[threadIdx.x] = 0; S.ivufirst[threadIdx.x] = -1; S.ivpre[threadIdx.x] = 0.0; }
+    __syncthreads();
+    for (long long i = threadIdx.x; i < src_cnt; i += kThreads) {
+        const uint32_t key = __ldcg(buf + i);
+        if (find_new_interval(S, key) >= 0) {
+            const int pos = atomicAdd(&S.n_keys, 1);
+            if (pos < kSmallN) skeys[pos] = key;
+        }
+    }
+    __syncthreads();
+    const int c = S.n_keys < kSmallN ? S.n_keys : kSmallN;
+    int P = 1;
+    while (P < c) P <<= 1;
+    for (int i = c + threadIdx.x; i < kSmallN; i += kThreads) skeys[i] = 0xffffffffu;
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < P; i += kThreads) {
+                const int ixj = i ^ j;
+                if (ixj > i) {
+                    const uint32_t a = skeys[i], b = skeys[ixj];
+                    const bool up = (i & k) == 0;
+                    if ((a > b) == up) { skeys[i] = b; skeys[ixj] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    // pass 1: run starts and value sums of this thread's kPer consecutive sorted elements
+    const int base = threadIdx.x * kPer;
+    uint32_t k[kPer];
+    unsigned long long lu = 0;
+    double ls = 0.0;
+    uint32_t prev = (base > 0 && base <= c) ? skeys[base - 1] : 0u;
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) {
+        const int i = base + e;
+        k[e] = (i < c) ? skeys[i] : 0xffffffffu;
+        if (i < c) {
+            const bool flag = (i == 0) || (k[e] != (e == 0 ? prev : k[e - 1]));
+            lu += flag ? 1 : 0;
+            ls += (double)sel_key_to_float(k[e]);
+        }
+    }
+    unsigned long long ubase = lu, tu;
+    double sbase = ls, tsum;
+    block_excl_scan(ubase, sbase, S.sc, S.ss, tu, tsum);
+    if (threadIdx.x == 0) S.n_unique = (int)tu;
+    // pass 2: first element of every interval
+    {
+        int nf = 0;
+        double run = sbase;
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) {
+            const int i = base + e;
+            if (i < c) {
+                const uint32_t pk = (e == 0) ? prev : k[e - 1];
+                const bool flag = (i == 0) || (k[e] != pk);
+                if (flag) {
+                    const int j = find_new_interval(S, k[e]);
+                    const int jp = (i == 0) ? -2 : find_new_interval(S, pk);
+                    if (j >= 0 && j != jp) {
+                        S.ivstart[j] = i;
+                        S.ivpre[j] = run;
+                        S.ivufirst[j] = (int)ubase + nf;
+                    }
+                    ++nf;
+                }
+                run += (double)sel_key_to_float(k[e]);
+            }
+        }
+    }
+    __syncthreads();
+    // pass 3: explicit cells (slot = unique index + interval index) and the end slot of every interval
+    {
+        int nf = 0;
+        double run = sbase;
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) {
+            const int i = base + e;
+            if (i < c) {
+                const uint32_t pk = (e == 0) ? prev : k[e - 1];
+                const bool flag = (i == 0) || (k[e] != pk);
+                const int j = find_new_interval(S, k[e]);
+                const double val = (double)sel_key_to_float(k[e]);
+                if (flag) {
+                    const int u = (int)ubase + nf;
+                    xkeys[u] = k[e];
+                    if (j >= 0) {
+                        xcpre[u + j] = (uint32_t)(S.niv[j].cbefore + (long long)(i - S.ivstart[j]));
+                        xspre[u + j] = S.niv[j].sbefore + (run - S.ivpre[j]);
+                    }
+                    ++nf;
+                }
+                const uint32_t nk = (i + 1 < c) ? ((e + 1 < kPer) ? k[e + 1] : skeys[i + 1]) : 0u;
+                const bool last_of_iv = (i + 1 >= c) || (find_new_interval(S, nk) != j);
+                if (last_of_iv && j >= 0) {
+                    const int u = (int)ubase + nf - 1;
+                    xcpre[u + 1 + j] = (uint32_t)(S.niv[j].cbefore + (long long)(i + 1 - S.ivstart[j]));
+                    xspre[u + 1 + j] = S.niv[j].sbefore + ((run + val) - S.ivpre[j]);
+                    S.niv[j].ncell = u - S.ivufirst[j] + 1;
+                }
+                run += val;
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int stbits = 0;
+        int next = S.n_unique;
+        for (int j = S.nm - 1; j >= 0; --j) {
+            if (S.ivufirst[j] < 0) {  // no element left in this interval: only its end slot
+                S.niv[j].ncell = 0;
+                xcpre[next + j] = (uint32_t)S.niv[j].cbefore;
+                xspre[next + j] = S.niv[j].sbefore;
+            } else {
+                next = S.ivufirst[j];
+            }
+        }
+        int cb = 0;
+        for (int j = 0; j < S.nm; ++j) { S.niv[j].sh = 0; S.niv[j].cellbase = cb; cb += S.niv[j].ncell; }
+        SolverView xv;
+        xv.xkeys = xkeys; xv.cpre = xcpre; xv.spre = xspre; xv.iv = S.niv; xv.m = S.nm;
+        xv.n = S.view.n; xv.stot = S.view.stot;
+        sel_init_slots(xv);
+        int ra[kMaxLv], rb[kMaxLv];
+        int open = (S.n_keys > kSmallN) ? -1 : sel_orq_pass(xv, s, S.lv, ra, rb);
+        if (open == 0) {
+            for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = sel_key_to_float(S.lv[q].key);
+        } else {
+            stbits = OGQ_ST_INTERNAL;
+            for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
+        }
+        if (stbits) status[t] |= stbits;
+        st->done = 1;
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+// Runs one solver pass for tensor t after all of its pieces of the current round arrived.
+// Called by every thread of the CTA; returns true when the tensor is finished.
+__device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long long* glsum, int scheme,
+                             int s, float* __restrict__ levels, int32_t* __restrict__ status,
+                             unsigned* nitems, int2* items, const uint32_t* round_buf, unsigned char* smem,
+                             SolverShared& S)
+{
+    uint32_t* cpre = reinterpret_cast<uint32_t*>(smem);
+    double* spre = reinterpret_cast<double*>(smem + ((kSlots * sizeof(uint32_t) + 15) / 16) * 16);
+    const bool pb = scheme == OGQ_BINGRAD_PB;
+    const int round = st->round;
+
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        S.view.m = st->m;
+        for (int j = 0; j < st->m; ++j) S.iv[j] = st->iv[j];
+        S.view.iv = S.iv;
+        S.view.xkeys = nullptr;
+        S.view.cpre = cpre;
+        S.view.spre = spre;
+        S.view.n = st->n;
+        sel_init_slots(S.view);
+        S.done = 0; S.nm = 0; S.internal = 0;
+        S.pb_a = -1; S.pb_b = -1; S.pb_c = -1;
+    }
+    __syncthreads();
+
+    // prefix arrays, interval by interval
+    for (int j = 0; j < S.view.m; ++j) {
+        const Interval iv = S.iv[j];
+        const int per = (iv.ncell + kThreads - 1) / kThreads;
+        const int c0 = threadIdx.x * per;
+        int c1 = c0 + per;
+        if (c1 > iv.ncell) c1 = iv.ncell;
+        unsigned long long lc = 0;
+        double ls = 0.0;
+        for (int c = c0; c < c1; ++c) {
+            const unsigned long long cn = __ldcg(gcnt + iv.cellbase + c);
+            const unsigned long long lsum = __ldcg(glsum + iv.cellbase + c);
+            lc += cn;
+            ls += sel_cell_sum(iv.klo + ((uint32_t)c << iv.sh), iv.sh, cn, lsum);
+        }
+        unsigned long long tc;
+        double ts;
+        block_excl_scan(lc, ls, S.sc, S.ss, tc, ts);
+        unsigned long long bc = (unsigned long long)iv.cbefore;
+        double bs = iv.sbefore;
+        if (round == 1 && j > 0) {  // round-1 intervals tile the key line: chain them
+            bc = cpre[S.view.slotbase[j] - 1];
+            bs = spre[S.view.slotbase[j] - 1];
+        }
+        unsigned long long rc = bc + lc;
+        double rs = bs + ls;
+        const int sb = S.view.slotbase[j];
+        for (int c = c0; c < c1; ++c) {
+            cpre[sb + c] = (uint32_t)rc;
+            spre[sb + c] = rs;
+            const unsigned long long cn = __ldcg(gcnt + iv.cellbase + c);
+            const unsigned long long lsum = __ldcg(glsum + iv.cellbase + c);
+            rc += cn;
+            rs += sel_cell_sum(iv.klo + ((uint32_t)c << iv.sh), iv.sh, cn, lsum);
+        }
+        if (threadIdx.x == 0) {
+            cpre[sb + iv.ncell] = (uint32_t)(bc + tc);
+            spre[sb + iv.ncell] = bs + ts;
+            if (round == 1) { S.iv[j].cbefore = (long long)bc; S.iv[j].sbefore = bs; }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && round == 1) {
+        st->stot = spre[S.view.nslots - 1];
+        if ((long long)cpre[S.view.nslots - 1] != st->n) S.internal = 1;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) S.view.stot = st->stot;
+    __syncthreads();
+
+    if (pb && !S.internal && S.view.stot > 0.0) {
+        // bracket of the sign change of g, evaluated at the lower edge of every cell
+        int a = -1, b = -1, cs = -1;
+        for (int sl = threadIdx.x; sl < S.view.nslots; sl += kThreads) {
+            if (sel_is_end_slot(S.view, sl)) continue;
+            double x;
+            const double g = sel_pb_g(S.view, sl, &x);
+            if (!(x < INFINITY)) continue;
+            const double eps = 1e-11 * (x * (double)S.view.n + S.view.stot);
+            if (g < -eps) a = sl;
+            if (g <= eps) b = sl;
+            if (g <= 0.0) cs = sl;
+        }
+        if (a >= 0) atomicMax(&S.pb_a, a);
+        if (b >= 0) atomicMax(&S.pb_b, b);
+        if (cs >= 0) atomicMax(&S.pb_c, cs);
+    }
+    __syncthreads();
+
+    if (threadIdx.x == 0) {
+        int ra[kMaxLv], rb[kMaxLv];
+        int open = 0;
+        int stbits = 0;
+        if (S.internal) {
+            stbits = OGQ_ST_INTERNAL;
+            S.done = 1;
+        } else if (pb) {
+            if (!(S.view.stot > 0.0)) {
+                levels[2 * t] = 0.f; levels[2 * t + 1] = 0.f;
+                stbits = OGQ_ST_CONSTANT;
+                S.done = 1;
+            } else {
+                int a = S.pb_a < 0 ? 0 : S.pb_a;
+                int b = S.pb_b < a ? a : S.pb_b;
+                int cs = S.pb_c < a ? a : S.pb_c;
+                if (cs > b) cs = b;
+                bool fine = true;
+                for (int sl = a; sl <= b; ++sl)
+                    if (!sel_is_end_slot(S.view, sl) && sel_slot_shift(S.view, sl) != 0) fine = false;
+                if (fine && !sel_is_end_slot(S.view, cs)) {
+                    const float b1 = (float)sel_pb_final(S.view, cs);
+                    levels[2 * t] = -b1; levels[2 * t + 1] = b1;
+                    S.done = 1;
+                } else {
+                    ra[0] = a; rb[0] = b; open = 1;
+                }
+            }
+        } else {
+            if (round == 1) {
+                for (int q = 0; q < s; ++q) S.lv[q].exact = 0;
+                LvInfo& l0 = S.lv[0];
+                l0.exact = 1; l0.key = ~__ldcg(&st->kmin_inv); l0.val = (double)sel_key_to_float(l0.key);
+                l0.c_lt = 0; l0.s_lt = 0.0; l0.c_le = 0; l0.s_le = 0.0;
+                LvInfo& l1 = S.lv[s - 1];
+                l1.exact = 1; l1.key = __ldcg(&st->kmax); l1.val = (double)sel_key_to_float(l1.key);
+                l1.c_lt = 0; l1.s_lt = 0.0; l1.c_le = st->n; l1.s_le = st->stot;
+            } else {
+                for (int q = 0; q < s; ++q) {
+                    const ExactLv& e = st->lv[q];
+                    S.lv[q].exact = e.exact;
+                    S.lv[q].key = e.key;
+                    S.lv[q].val = (double)sel_key_to_float(e.key);
+                    S.lv[q].c_lt = e.c_lt; S.lv[q].c_le = e.c_le; S.lv[q].s_lt = e.s_lt; S.lv[q].s_le = e.s_le;
+                }
+            }
+            open = sel_orq_pass(S.view, s, S.lv, ra, rb);
+            if (open < 0) {
+                stbits = OGQ_ST_INTERNAL;
+                S.done = 1;
+            } else if (open == 0) {
+                for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = sel_key_to_float(S.lv[q].key);
+                S.done = 1;
+            } else {
+                for (int q = 0; q < s; ++q) {
+                    ExactLv& e = st->lv[q];
+                    e.exact = S.lv[q].exact; e.key = S.lv[q].key;
+                    e.c_lt = S.lv[q].c_lt; e.c_le = S.lv[q].c_le; e.s_lt = S.lv[q].s_lt; e.s_le = S.lv[q].s_le;
+                }
+            }
+        }
+        if (!S.done) {
+            S.cand = 0;
+            const int nm = (round + 1 > kMaxRounds) ? -2 : sel_refine(S.view, open, ra, rb, !pb, S.niv, &S.cand);
+            if (nm < 0) {
+                stbits = (nm == -2) ? OGQ_ST_ITER_CAP : OGQ_ST_INTERNAL;
+                S.done = 1;
+            } else {
+                S.nm = nm;
+            }
+        }
+        if (S.done && stbits) {
+            // unresolved: leave zeros rather than garbage
+            if (pb) { levels[2 * t] = 0.f; levels[2 * t + 1] = 0.f; }
+            else for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
+        }
+        if (stbits) status[t] |= stbits;
+    }
+    __syncthreads();
+
+    if (S.done) {
+        if (threadIdx.x == 0) { st->done = 1; __threadfence(); }
+        return true;
+    }
+    if (!pb && round >= 2 && S.cand <= kSmallN && round_buf != nullptr) {
+        const long long src_cnt = (long long)__ldcg(&st->cursor[round & 1]);
+        if (src_cnt <= kSortScanMax) {
+            sort_finish(st, t, s, round_buf, src_cnt, levels, status, smem, S);
+            return true;
+        }
+    }
+    // prepare the next round: clear the cells it will use, publish the new intervals
+    const int ncells_next = S.niv[S.nm - 1].cellbase + S.niv[S.nm - 1].ncell;
+    for (int i = threadIdx.x; i < ncells_next; i += kThreads) {
+        gcnt[i] = 0u;
+        glsum[i] = 0ull;
+    }
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < S.nm; ++j) st->iv[j] = S.niv[j];
+        st->m = S.nm;
+        st->round = round + 1;
+        st->arrive = 0;
+        const int next = round + 1;
+        st->cursor[next & 1] = 0ull;  // buffer the next round writes
+        if (next == 3) {
+            const unsigned long long cntk = __ldcg(&st->cursor[0]);
+            unsigned ns = (unsigned)((cntk + kSliceElems - 1) / kSliceElems);
+            if (ns < 1) ns = 1;
+            if (ns > kMaxSlices) ns = kMaxSlices;
+            st->expected = ns;
+            const unsigned base = atomicAdd(nitems, ns);
+            for (unsigned i = 0; i < ns; ++i) items[base + i] = make_int2(t, (int)i);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    return false;
+}
+
+// ---------------------------------------------------------------------------
+// Small tensors: sort the keys in shared memory and apply the definitions directly.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ int lower_bound_u32(const uint32_t* a, int n, uint32_t k)
+{
+    int lo = 0, hi = n;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] < k) lo = mid + 1; else hi = mid; }
+    return lo;
+}
+
+__device__ __forceinline__ int upper_bound_u32(const uint32_t* a, int n, uint32_t k)
+{
+    int lo = 0, hi = n;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] <= k) lo = mid + 1; else hi = mid; }
+    return lo;
+}
+
+__device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, int t, int scheme, int s,
+                             float* __restrict__ levels, int32_t* __restrict__ status, TState* st,
+                             unsigned char* smem)
+{
+    __shared__ double sh_d[kWarps];
+    __shared__ uint32_t sh_lvkey[kMaxLv];
+    __shared__ int sh_flag;
+    __shared__ double sh_bcast;
+    uint32_t* keys = reinterpret_cast<uint32_t*>(smem);
+    const bool pb = scheme == OGQ_BINGRAD_PB;
+    int P = 1;
+    while (P < n) P <<= 1;
+    if (threadIdx.x == 0) sh_flag = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < P; i += kThreads) {
+        uint32_t key = 0xffffffffu;
+        if (i < n) {
+            uint32_t bits = __float_as_uint(__ldg(grad + tb + i));
+            if ((bits & 0x7f800000u) == 0x7f800000u) sh_flag = 1;
+            if (pb) key = bits | 0x80000000u;
+            else {
+                if (bits == 0x80000000u) bits = 0u;
+                key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+            }
+        }
+        keys[i] = key;
+    }
+    __syncthreads();
+    // bitonic sort, ascending
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < P; i += kThreads) {
+                const int ixj = i ^ j;
+                if (ixj > i) {
+                    const uint32_t a = keys[i], b = keys[ixj];
+                    const bool up = (i & k) == 0;
+                    if ((a > b) == up) { keys[i] = b; keys[ixj] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    int stbits = 0;
+    if (sh_flag) {
+        if (threadIdx.x == 0) {
+            const int nl = pb ? 2 : s;
+            for (int q = 0; q < nl; ++q) levels[(int64_t)t * nl + q] = 0.f;
+            status[t] = OGQ_ST_NONFINITE;
+            st->done = 1;
+        }
+        return;
+    }
+    if (!pb) {
+        if (keys[0] == keys[n - 1]) stbits |= OGQ_ST_CONSTANT;
+        if (threadIdx.x == 0) {
+            for (int q = 0; q < s; ++q) sh_lvkey[q] = keys[0];
+            sh_lvkey[s - 1] = keys[n - 1];
+        }
+        __syncthreads();
+        for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
+            for (int q = stride; q < s - 1; q += 2 * stride) {
+                const uint32_t kl = sh_lvkey[q - stride], kr = sh_lvkey[q + stride];
+                uint32_t res = kl;
+                if (kr > kl) {
+                    const int i0 = lower_bound_u32(keys, n, kl), i1 = upper_bound_u32(keys, n, kr);
+                    const double Lv = (double)sel_key_to_float(kl), Rv = (double)sel_key_to_float(kr);
+                    double a = 0.0;
+                    for (int i = i0 + threadIdx.x; i < i1; i += kThreads) a += (double)sel_key_to_float(keys[i]) - Lv;
+                    a = block_sum(a, sh_d);
+                    if (threadIdx.x == 0) sh_bcast = a;
+                    __syncthreads();
+                    a = sh_bcast;
+                    const double T = a / (Rv - Lv);
+                    long long k = (long long)floor(T);
+                    const long long m = i1 - i0;
+                    if (k < 0) k = 0;
+                    if (k > m - 1) k = m - 1;
+                    res = keys[i1 - 1 - (int)k];
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) sh_lvkey[q] = res;
+                __syncthreads();
+            }
+        }
+        if (threadIdx.x < s) levels[(int64_t)t * s + threadIdx.x] = sel_key_to_float(sh_lvkey[threadIdx.x]);
+        if (threadIdx.x == 0) { status[t] = stbits; st->done = 1; }
+        return;
+    }
+    // BinGrad-pb: prefix sums of the sorted magnitudes, then the sign change of g
+    double* pre = reinterpret_cast<double*>(smem + kSmallN * sizeof(uint32_t));  // [n + 1]
+    __shared__ unsigned long long sc_[kWarps];
+    __shared__ double ss_[kWarps];
+    __shared__ int sh_c;
+    const int per = (n + kThreads - 1) / kThreads;
+    const int c0 = threadIdx.x * per < n ? threadIdx.x * per : n;
+    const int c1 = c0 + per < n ? c0 + per : n;
+    unsigned long long dummy = 0, dt;
+    double ls = 0.0, tot;
+    for (int i = c0; i < c1; ++i) ls += (double)sel_key_to_float(keys[i]);
+    block_excl_scan(dummy, ls, sc_, ss_, dt, tot);
+    double run = ls;
+    for (int i = c0; i < c1; ++i) { pre[i] = run; run += (double)sel_key_to_float(keys[i]); }
+    if (threadIdx.x == 0) { pre[n] = tot; sh_c = -1; }
+    __syncthreads();
+    int best = -1;
+    for (int i = threadIdx.x; i < n; i += kThreads) {
+        const double x = (double)sel_key_to_float(keys[i]);
+        const int first = lower_bound_u32(keys, n, keys[i]);
+        const double g = x * (double)n - (tot - pre[first]);
+        if (g <= 0.0) best = i;
+    }
+    if (best >= 0) atomicMax(&sh_c, best);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float b1 = 0.f;
+        if (!(tot > 0.0)) stbits |= OGQ_ST_CONSTANT;
+        else {
+            const int c = sh_c < 0 ? 0 : sh_c;
+            const double x = (double)sel_key_to_float(keys[c]);
+            const int up = upper_bound_u32(keys, n, keys[c]);
+            const double stat_up = (tot - pre[up]) / (double)n;
+            b1 = (float)(stat_up > x ? stat_up : x);
+        }
+        levels[2 * t] = -b1; levels[2 * t + 1] = b1;
+        status[t] = stbits;
+        st->done = 1;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Kernels
+// ---------------------------------------------------------------------------
+struct SelArgs {
+    const float* grad;
+    const int64_t* off;
+    int T;
+    int64_t total, chunk;
+    int flat_ctas, scheme, s;
+    float* levels;
+    int32_t* status;
+    SelWs ws;
+};
+
+// Continues the rounds of one tensor on a single CTA until it is finished (the working set is
+// tiny by then).  Called by the CTA that completed round >= 3.
+__device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table& tb, SolverShared& S)
+{
+    TState* st = A.ws.st + t;
+    uint32_t* gcnt = A.ws.gcnt + (size_t)t * kCells;
+    unsigned long long* glsum = A.ws.glsum + (size_t)t * kCells;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
+    const int64_t tbeg = __ldg(A.off + t);
+    for (int guard = 0; guard < kMaxRounds; ++guard) {
+        const int round = st->round;
+        const uint32_t* src = A.ws.buf[(round - 1) & 1];  // 16-byte aligned base; indices are absolute
+        const int64_t cnt = (int64_t)__ldcg(&st->cursor[(round - 1) & 1]);
+        __syncthreads();
+        if (threadIdx.x == 0) table_from_intervals(tb, st->iv, st->m);
+        __syncthreads();
+        zero_hist(hist, tb.ncells);
+        __syncthreads();
+        Stager stg;
+        stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+        stg.dst = A.ws.buf[round & 1] + tbeg;
+        stg.cursor = &st->cursor[round & 1];
+        stg.fill = 0;
+        uint32_t kmin = 0, kmax = 0, nf = 0;
+        stream_piece<false, false, true>(src, tbeg, tbeg + cnt, false, tb, hist, hist + kCells, hist + 2 * kCells,
+                                         stg, kmin, kmax, nf);
+        stg.flush();
+        __syncthreads();
+        flush_hist(hist, tb.ncells, gcnt, glsum);
+        __threadfence();
+        __syncthreads();
+        if (solver_round(st, t, gcnt, glsum, A.scheme, A.s, A.levels, A.status, A.ws.nitems, A.ws.items,
+                         A.ws.buf[round & 1] + tbeg, smem, S))
+            return;
+    }
+    if (threadIdx.x == 0) {
+        A.status[t] |= OGQ_ST_ITER_CAP;
+        st->done = 1;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ Table tb;
+    __shared__ SolverShared S;
+    __shared__ Interval r1iv[kMaxIv];
+    __shared__ int sh_i[kWarps];
+    __shared__ uint32_t sh_u[2 * kWarps];
+    __shared__ int sh_last;
+    const bool pb = A.scheme == OGQ_BINGRAD_PB;
+    const int nl = pb ? 2 : A.s;
+
+    if ((int)blockIdx.x >= A.flat_ctas) {
+        // one extra CTA per tensor: empty and small tensors are settled here
+        const int t = blockIdx.x - A.flat_ctas;
+        const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
+        const int64_t n = tend - tbeg;
+        if (n <= 0) {
+            if (threadIdx.x < nl) A.levels[(int64_t)t * nl + threadIdx.x] = 0.f;
+            if (threadIdx.x == 0) { A.status[t] = OGQ_ST_EMPTY; A.ws.st[t].done = 1; }
+        } else if (n <= kSmallN) {
+            small_tensor(A.grad, tbeg, (int)n, t, A.scheme, A.s, A.levels, A.status, A.ws.st + t, smem);
+        }
+        return;
+    }
+
+    const int64_t lo = (int64_t)blockIdx.x * A.chunk;
+    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
+
+    for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+        const int64_t n = tend - tbeg;
+        if (n <= kSmallN) return;
+        TState* st = A.ws.st + t;
+        // anchor of the fine window: largest binade among 256 strided samples, plus two
+        int e = 0;
+        {
+            const int64_t idx = tbeg + (int64_t)threadIdx.x * n / kThreads;
+            e = (int)((__float_as_uint(__ldg(A.grad + idx)) >> 23) & 255u);
+            if (e == 255) e = 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) { const int x = __shfl_xor_sync(0xffffffffu, e, o); e = x > e ? x : e; }
+        }
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) sh_i[threadIdx.x >> 5] = e;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int mx = 0;
+            for (int w = 0; w < kWarps; ++w) mx = sh_i[w] > mx ? sh_i[w] : mx;
+            int hi_e = mx + 2;
+            if (hi_e < kSelW) hi_e = kSelW;
+            if (hi_e > 256) hi_e = 256;
+            const int m = round1_intervals(hi_e, pb, r1iv);
+            table_from_intervals(tb, r1iv, m);
+        }
+        __syncthreads();
+        zero_hist(hist, tb.ncells);
+        __syncthreads();
+        Stager stg;
+        stg.stage = nullptr; stg.dst = nullptr; stg.cursor = nullptr; stg.fill = 0;
+        uint32_t kmin = 0xffffffffu, kmax = 0u, nf = 0u;
+        stream_piece<true, true, false>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stg,
+                                        kmin, kmax, nf);
+        // combine min / max / non-finite over the CTA, then one atomic each
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const uint32_t a = __shfl_xor_sync(0xffffffffu, kmin, o), b = __shfl_xor_sync(0xffffffffu, kmax, o);
+            kmin = a < kmin ? a : kmin;
+            kmax = b > kmax ? b : kmax;
+            nf |= __shfl_xor_sync(0xffffffffu, nf, o);
+        }
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) {
+            sh_u[threadIdx.x >> 5] = kmin;
+            sh_u[kWarps + (threadIdx.x >> 5)] = kmax;
+            if (nf) atomicOr(&st->nonfinite, 1u);
+        }
+        __syncthreads();
+        flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+        if (threadIdx.x == 0) {
+            uint32_t mn = 0xffffffffu, mx = 0u;
+            for (int w = 0; w < kWarps; ++w) { mn = sh_u[w] < mn ? sh_u[w] : mn; mx = sh_u[kWarps + w] > mx ? sh_u[kWarps + w] : mx; }
+            atomicMax(&st->kmin_inv, ~mn);
+            atomicMax(&st->kmax, mx);
+        }
+        __threadfence();
+        __syncthreads();
+        const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
+        if (threadIdx.x == 0) {
+            const unsigned prev = atomicAdd(&st->arrive, 1u);
+            sh_last = (prev == (unsigned)(c1 - c0));
+        }
+        __syncthreads();
+        if (!sh_last) return;
+        __threadfence();
+        // last CTA of this tensor: set up the state and run the first solver pass
+        if (threadIdx.x == 0) {
+            st->n = n;
+            st->round = 1;
+            st->m = tb.m;
+            for (int j = 0; j < tb.m; ++j) st->iv[j] = r1iv[j];
+            int stb = 0;
+            const uint32_t kmn = ~__ldcg(&st->kmin_inv), kmx = __ldcg(&st->kmax);
+            if (__ldcg(&st->nonfinite)) stb |= OGQ_ST_NONFINITE;
+            else if (!pb && kmn == kmx) stb |= OGQ_ST_CONSTANT;
+            A.status[t] = stb;
+            sh_last = stb;
+            if (stb & OGQ_ST_NONFINITE) {
+                for (int q = 0; q < nl; ++q) A.levels[(int64_t)t * nl + q] = 0.f;
+                st->done = 1;
+            } else if (stb & OGQ_ST_CONSTANT) {
+                const float v = sel_key_to_float(kmn);
+                for (int q = 0; q < nl; ++q) A.levels[(int64_t)t * nl + q] = v;
+                st->done = 1;
+            }
+        }
+        __syncthreads();
+        if (sh_last & (OGQ_ST_NONFINITE | OGQ_ST_CONSTANT)) return;
+        solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
+                     A.levels, A.status, A.ws.nitems, A.ws.items, nullptr, smem, S);
+    });
+}
+
+__global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ Table tb;
+    __shared__ SolverShared S;
+    __shared__ int sh_last;
+    const bool pb = A.scheme == OGQ_BINGRAD_PB;
+    const int64_t lo = (int64_t)blockIdx.x * A.chunk;
+    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
+
+    for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+        const int64_t n = tend - tbeg;
+        if (n <= kSmallN) return;
+        TState* st = A.ws.st + t;
+        if (__ldcg(&st->done)) return;
+        __syncthreads();
+        if (threadIdx.x == 0) table_from_intervals(tb, st->iv, __ldcg(&st->m));
+        __syncthreads();
+        zero_hist(hist, tb.ncells);
+        __syncthreads();
+        Stager stg;
+        stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+        stg.dst = A.ws.buf[0] + tbeg;
+        stg.cursor = &st->cursor[0];
+        stg.fill = 0;
+        uint32_t kmin = 0, kmax = 0, nf = 0;
+        stream_piece<false, true, true>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stg,
+                                        kmin, kmax, nf);
+        stg.flush();
+        __syncthreads();
+        flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+        __threadfence();
+        __syncthreads();
+        const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
+        if (threadIdx.x == 0) {
+            const unsigned prev = atomicAdd(&st->arrive, 1u);
+            sh_last = (prev == (unsigned)(c1 - c0));
+        }
+        __syncthreads();
+        if (!sh_last) return;
+        __threadfence();
+        solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
+                     A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, smem, S);
+    });
+}
+
+__global__ void __launch_bounds__(kThreads) k_sel_round3(SelArgs A)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ Table tb;
+    __shared__ SolverShared S;
+    __shared__ int sh_last;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
+    const unsigned nitems = __ldcg(A.ws.nitems);
+
+    for (unsigned w = blockIdx.x; w < nitems; w += gridDim.x) {
+        const int2 it = A.ws.items[w];
+        const int t = it.x;
+        TState* st = A.ws.st + t;
+        const int64_t tbeg = __ldg(A.off + t);
+        const unsigned ns = __ldcg(&st->expected);
+        const int64_t cnt = (int64_t)__ldcg(&st->cursor[0]);
+        int64_t per = (cnt + ns - 1) / ns;
+        per = (per + 3) & ~(int64_t)3;
+        int64_t pb_ = per * it.y, pe_ = pb_ + per;
+        if (pb_ > cnt) pb_ = cnt;
+        if (pe_ > cnt) pe_ = cnt;
+        __syncthreads();
+        if (threadIdx.x == 0) table_from_intervals(tb, st->iv, __ldcg(&st->m));
+        __syncthreads();
+        zero_hist(hist, tb.ncells);
+        __syncthreads();
+        Stager stg;
+        stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+        stg.dst = A.ws.buf[1] + tbeg;
+        stg.cursor = &st->cursor[1];
+        stg.fill = 0;
+        uint32_t kmin = 0, kmax = 0, nf = 0;
+        stream_piece<false, false, true>(A.ws.buf[0], tbeg + pb_, tbeg + pe_, false, tb, hist, hist + kCells,
+                                         hist + 2 * kCells, stg, kmin, kmax, nf);
+        stg.flush();
+        __syncthreads();
+        flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const unsigned prev = atomicAdd(&st->arrive, 1u);
+            sh_last = (prev == ns - 1);
+        }
+        __syncthreads();
+        if (!sh_last) continue;
+        __threadfence();
+        if (!solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
+                          A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[1] + tbeg, smem, S))
+            finish_alone(A, t, smem, tb, S);
+    }
+}
+
+cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int T, int64_t total, int scheme,
+                                 int s, float* d_levels, int32_t* d_status, void* d_ws, size_t /*ws_bytes*/,
+                                 int sm_count, cudaStream_t stream)
+{
+    {
+        cudaError_t e;
+        e = cudaFuncSetAttribute(k_sel_round1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(k_sel_round2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+    }
+    int target = sm_count * 2 < kMaxFlatCtas ? sm_count * 2 : kMaxFlatCtas;
+    FlatGrid g = make_flat_grid(total, target, 16384);
+    SelArgs A;
+    A.grad = d_grad; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
+    A.scheme = scheme; A.s = s; A.levels = d_levels; A.status = d_status;
+    A.ws = sel_carve(d_ws, T, total);
+    cudaError_t e = cudaMemsetAsync(d_ws, 0, sel_zero_bytes(T), stream);
+    if (e != cudaSuccess) return e;
+    k_sel_round1<<<g.ctas + T, kThreads, kSmemBytes, stream>>>(A);
+    k_sel_round2<<<g.ctas, kThreads, kSmemBytes, stream>>>(A);
+    k_sel_round3<<<sm_count * 2, kThreads, kSmemBytes, stream>>>(A);
+    return cudaGetLastError();
+}
+
+}  // namespace ogq
