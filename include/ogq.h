@@ -14,7 +14,8 @@
  *     h_* are HOST pointers.  d_grad, d_out and every packed buffer must be
  *     16-byte aligned; tensor offsets need no alignment (tensors whose offset
  *     is not a multiple of 4 elements take a scalar-load path).
- *   - The library allocates no memory and keeps no state between calls.  Scratch
+ *   - The library allocates no memory and keeps no state between calls on the data
+ *     path (only the measurement helpers at the end keep host-side records).  Scratch
  *     memory is the caller's `d_ws` of at least ogq_workspace_bytes(...) bytes,
  *     256-byte aligned; its contents need not be preserved or initialised.
  *   - Calls only enqueue work on `stream` and return at once.  The return code
@@ -134,6 +135,22 @@ ogq_status ogq_quantize_pack(const float *d_grad, const int64_t *d_off, int T, i
 ogq_status ogq_unpack_sum(const uint32_t *const *d_packed_k, const float *const *d_levels_k, int K,
                           const int64_t *d_off, const int64_t *d_packed_off, int T, int64_t total_elems,
                           int s, float scale, float *d_out, ogq_stream_t stream);
+
+/*
+ * Measurement helpers (no counterpart in the paper; they do not touch the data path).
+ * ogq_launch_count: number of kernels this library has launched in this process so far.
+ * ogq_profile_enable(1): from now on every kernel launch of the library is bracketed by two CUDA
+ *   events recorded on the launch stream; ogq_profile_enable(0) stops recording.  Turning it on
+ *   discards earlier records.  Process-wide and not thread-safe: use it from one thread, around
+ *   whole calls, and never while a stream is being captured.
+ * ogq_profile_collect: waits for the recorded events, then writes up to max_records entries:
+ *   h_ms[i] is the device time of launch i in milliseconds and h_names receives the kernel
+ *   names, each padded to name_stride bytes (NUL terminated).  Returns the number of records
+ *   written and clears them.
+ */
+unsigned long long ogq_launch_count(void);
+int ogq_profile_enable(int on);
+int ogq_profile_collect(float *h_ms, char *h_names, int name_stride, int max_records);
 
 #ifdef __cplusplus
 }

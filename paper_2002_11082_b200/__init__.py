@@ -26,5 +26,8 @@ from .binding import (  # noqa: F401
     ogq_levels_orq,
     ogq_quantize_pack,
     ogq_unpack_sum,
+    ogq_launch_count,
+    ogq_profile_enable,
+    ogq_profile_collect,
     device_pointer_array,
 )

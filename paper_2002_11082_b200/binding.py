@@ -56,6 +56,12 @@ def lib() -> ctypes.CDLL:
         L.ogq_quantize_pack.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, ctypes.c_uint64, ctypes.c_uint32, vp, vp, vp]
         L.ogq_unpack_sum.restype = i32
         L.ogq_unpack_sum.argtypes = [vp, vp, i32, vp, vp, i32, i64, i32, ctypes.c_float, vp, vp]
+        L.ogq_launch_count.restype = ctypes.c_ulonglong
+        L.ogq_launch_count.argtypes = []
+        L.ogq_profile_enable.restype = i32
+        L.ogq_profile_enable.argtypes = [i32]
+        L.ogq_profile_collect.restype = i32
+        L.ogq_profile_collect.argtypes = [vp, vp, i32, i32]
         _lib = L
     return _lib
 
@@ -141,6 +147,24 @@ def ogq_unpack_sum(d_packed_k, d_levels_k, K: int, d_off, d_packed_off, T: int, 
                              int(T), int(total_elems), int(s), float(scale), _ptr(d_out), _stream(stream)),
         "ogq_unpack_sum",
     )
+
+
+def ogq_launch_count() -> int:
+    return int(lib().ogq_launch_count())
+
+
+def ogq_profile_enable(on: bool) -> None:
+    lib().ogq_profile_enable(1 if on else 0)
+
+
+def ogq_profile_collect(max_records: int = 65536):
+    """Returns [(kernel name, milliseconds), ...] for the launches recorded since profiling was enabled."""
+    ms = np.zeros(max_records, dtype=np.float32)
+    stride = 48
+    names = ctypes.create_string_buffer(max_records * stride)
+    n = lib().ogq_profile_collect(ms.ctypes.data, ctypes.cast(names, ctypes.c_void_p), stride, max_records)
+    raw = names.raw
+    return [(raw[i * stride : (i + 1) * stride].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n)]
 
 
 def device_pointer_array(tensors: Sequence, device=None):

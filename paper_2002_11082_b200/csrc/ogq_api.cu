@@ -1,8 +1,40 @@
 // extern "C" entry points: argument validation, scratch layout, kernel launches.
 #include <cuda_runtime.h>
+#include <string.h>
+
+#include <vector>
 
 #include "../../include/ogq.h"
 #include "ogq_internal.h"
+
+namespace ogq {
+
+struct ProfRec {
+    const char* name;
+    cudaEvent_t a, b;
+};
+static std::vector<ProfRec> g_prof;
+static bool g_prof_on = false;
+static unsigned long long g_launches = 0;
+
+void launch_begin(const char* name, cudaStream_t stream)
+{
+    ++g_launches;
+    if (!g_prof_on) return;
+    ProfRec r;
+    r.name = name;
+    if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+    cudaEventRecord(r.a, stream);
+    g_prof.push_back(r);
+}
+
+void launch_end(cudaStream_t stream)
+{
+    if (!g_prof_on || g_prof.empty()) return;
+    cudaEventRecord(g_prof.back().b, stream);
+}
+
+}  // namespace ogq
 
 namespace {
 
@@ -23,6 +55,39 @@ bool valid_orq_levels(int s) { return s == 3 || s == 5 || s == 9 || s == 17; }
 extern "C" {
 
 const char* ogq_version(void) { return "ogq 0.1 (sm_100a)"; }
+
+unsigned long long ogq_launch_count(void) { return ogq::g_launches; }
+
+int ogq_profile_enable(int on)
+{
+    if (on) {
+        for (auto& r : ogq::g_prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+        ogq::g_prof.clear();
+    }
+    ogq::g_prof_on = on != 0;
+    return 0;
+}
+
+int ogq_profile_collect(float* h_ms, char* h_names, int name_stride, int max_records)
+{
+    int n = 0;
+    for (auto& r : ogq::g_prof) {
+        if (n < max_records && h_ms && cudaEventSynchronize(r.b) == cudaSuccess) {
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, r.a, r.b);
+            h_ms[n] = ms;
+            if (h_names && name_stride > 0) {
+                strncpy(h_names + (size_t)n * name_stride, r.name, (size_t)name_stride - 1);
+                h_names[(size_t)n * name_stride + name_stride - 1] = 0;
+            }
+            ++n;
+        }
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    ogq::g_prof.clear();
+    return n;
+}
 
 int ogq_bits_for_levels(int s)
 {

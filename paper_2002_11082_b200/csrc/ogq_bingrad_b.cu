@@ -136,8 +136,10 @@ cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, i
     cudaError_t e = cudaMemsetAsync(d_ws, 0, bb_ws_bytes(T, g.ctas), stream);
     if (e != cudaSuccess) return e;
     for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
+        launch_begin("k_bb_pass", stream);
         k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters,
                                                    d_levels, d_thresh, d_status, ws);
+        launch_end(stream);
     }
     return cudaGetLastError();
 }

@@ -201,6 +201,7 @@ cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int 
     k_quantize_pack<B, TH><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, s,     \
                                                             d_levels, d_thresh, slo, shi, stream_id, \
                                                             d_packed_off, d_packed)
+    launch_begin(scheme == OGQ_BINGRAD_B ? "k_quantize_pack_threshold" : "k_quantize_pack_random", stream);
     if (scheme == OGQ_BINGRAD_B) {
         OGQ_LAUNCH_Q(1, true);
     } else {
@@ -214,6 +215,7 @@ cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int 
         }
     }
 #undef OGQ_LAUNCH_Q
+    launch_end(stream);
     return cudaGetLastError();
 }
 
@@ -226,6 +228,7 @@ cudaError_t launch_unpack_sum(const uint32_t* const* d_packed_k, const float* co
 #define OGQ_LAUNCH_U(B)                                                                               \
     k_unpack_sum<B><<<g.ctas, kThreads, 0, stream>>>(d_packed_k, d_levels_k, K, d_off, d_packed_off, T, \
                                                      total, g.chunk, s, scale, d_out)
+    launch_begin("k_unpack_sum", stream);
     switch (bits) {
         case 1: OGQ_LAUNCH_U(1); break;
         case 2: OGQ_LAUNCH_U(2); break;
@@ -235,6 +238,7 @@ cudaError_t launch_unpack_sum(const uint32_t* const* d_packed_k, const float* co
         default: return cudaErrorInvalidValue;
     }
 #undef OGQ_LAUNCH_U
+    launch_end(stream);
     return cudaGetLastError();
 }
 

@@ -7,6 +7,10 @@
 
 namespace ogq {
 
+// Instrumentation: counts launches and, when profiling is on, brackets them with events.
+void launch_begin(const char* name, cudaStream_t stream);
+void launch_end(cudaStream_t stream);
+
 constexpr int kMaxFlatCtas = 4096;  // upper bound on CTAs of a flat streaming grid (scratch sizing)
 
 cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, int T, int64_t total,

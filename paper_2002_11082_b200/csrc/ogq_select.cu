@@ -1180,9 +1180,15 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     A.ws = sel_carve(d_ws, T, total);
     cudaError_t e = cudaMemsetAsync(d_ws, 0, sel_zero_bytes(T), stream);
     if (e != cudaSuccess) return e;
+    launch_begin("k_sel_round1", stream);
     k_sel_round1<<<g.ctas + T, kThreads, kSmemBytes, stream>>>(A);
+    launch_end(stream);
+    launch_begin("k_sel_round2", stream);
     k_sel_round2<<<g.ctas, kThreads, kSmemBytes, stream>>>(A);
+    launch_end(stream);
+    launch_begin("k_sel_round3", stream);
     k_sel_round3<<<sm_count * 2, kThreads, kSmemBytes, stream>>>(A);
+    launch_end(stream);
     return cudaGetLastError();
 }
 
