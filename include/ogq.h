@@ -41,7 +41,8 @@ typedef enum {
     OGQ_ERR_INVALID_ARG = 1,
     OGQ_ERR_UNSUPPORTED = 2,
     OGQ_ERR_WORKSPACE = 3,
-    OGQ_ERR_CUDA = 4
+    OGQ_ERR_CUDA = 4,
+    OGQ_ERR_LIMIT = 5 /* the request exceeds a fixed capacity of the entry point */
 } ogq_status;
 
 typedef enum { OGQ_BINGRAD_PB = 0, OGQ_BINGRAD_B = 1, OGQ_ORQ = 2 } ogq_scheme;
@@ -93,6 +94,31 @@ size_t ogq_workspace_bytes(int num_tensors, int64_t total_elems, int max_levels)
 ogq_status ogq_levels_bingrad(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems,
                               int variant, int lloyd_iters, float *d_levels, float *d_thresh,
                               int32_t *d_status, void *d_ws, size_t ws_bytes, ogq_stream_t stream);
+
+/*
+ * BinGrad-b levels without caller-provided scratch.  The paper has no counterpart; this exists
+ * for callers that must not allocate device memory: code that runs where the allocator is off
+ * limits (a plugin or communication hook invoked in the middle of a training step, a process
+ * whose memory pool is owned and fully reserved by another component, a strict real-time loop
+ * where cudaMalloc's implicit synchronisation is unacceptable) and that cannot size and keep an
+ * ogq_workspace_bytes() buffer either.  Same results as ogq_levels_bingrad(..., OGQ_BINGRAD_B,
+ * ...): the same kernels run, but their partial-sum slots and counters live in a fixed array
+ * inside the library image instead of d_ws.
+ *   - Capacity: at most OGQ_NOALLOC_MAX_TENSORS tensors per call (any element count).  More
+ *     returns OGQ_ERR_LIMIT and enqueues nothing.  The array costs every GPU that loads the
+ *     library about 304 KB of device memory until the process exits.
+ *   - The call allocates and frees nothing.  The first call on each device looks up the array's
+ *     device address (with that device current); make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one array.  The part a call uses is cleared on `stream`
+ *     before its kernels run, so leftovers of earlier calls do no harm, but two calls whose
+ *     work overlaps on the GPU (different streams, no ordering between them) race on it and
+ *     give wrong levels.  Order such calls, or use ogq_levels_bingrad with separate scratch.
+ */
+#define OGQ_NOALLOC_MAX_TENSORS 1024
+ogq_status ogq_levels_bingrad_b_noalloc(const float *d_grad, const int64_t *d_off, int T,
+                                        int64_t total_elems, int lloyd_iters, float *d_levels,
+                                        float *d_thresh, int32_t *d_status, ogq_stream_t stream);
 
 /*
  * ORQ levels (Algorithm 1 with the discrete form of the simplified optimal

@@ -23,6 +23,7 @@ from .binding import (  # noqa: F401
     ogq_packed_layout,
     ogq_workspace_bytes,
     ogq_levels_bingrad,
+    ogq_levels_bingrad_b_noalloc,
     ogq_levels_orq,
     ogq_quantize_pack,
     ogq_unpack_sum,

@@ -13,7 +13,8 @@ _LIB_PATH = os.path.join(_HERE, "libogq.so")
 OGQ_BINGRAD_PB, OGQ_BINGRAD_B, OGQ_ORQ = 0, 1, 2
 OGQ_ST_EMPTY, OGQ_ST_NONFINITE, OGQ_ST_CONSTANT, OGQ_ST_ITER_CAP, OGQ_ST_INTERNAL = 1, 2, 4, 8, 16
 
-_STATUS_NAMES = {1: "OGQ_ERR_INVALID_ARG", 2: "OGQ_ERR_UNSUPPORTED", 3: "OGQ_ERR_WORKSPACE", 4: "OGQ_ERR_CUDA"}
+_STATUS_NAMES = {1: "OGQ_ERR_INVALID_ARG", 2: "OGQ_ERR_UNSUPPORTED", 3: "OGQ_ERR_WORKSPACE", 4: "OGQ_ERR_CUDA",
+                 5: "OGQ_ERR_LIMIT"}
 
 
 class OgqError(RuntimeError):
@@ -50,6 +51,8 @@ def lib() -> ctypes.CDLL:
         L.ogq_workspace_bytes.argtypes = [i32, i64, i32]
         L.ogq_levels_bingrad.restype = i32
         L.ogq_levels_bingrad.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.ogq_levels_bingrad_b_noalloc.restype = i32
+        L.ogq_levels_bingrad_b_noalloc.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp]
         L.ogq_levels_orq.restype = i32
         L.ogq_levels_orq.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, sz, vp]
         L.ogq_quantize_pack.restype = i32
@@ -117,6 +120,19 @@ def ogq_levels_bingrad(d_grad, d_off, T: int, total_elems: int, variant: int, ll
                                  int(lloyd_iters), _ptr(d_levels), _ptr(d_thresh), _ptr(d_status),
                                  _ptr(d_ws), int(ws_bytes), _stream(stream)),
         "ogq_levels_bingrad",
+    )
+
+
+def ogq_levels_bingrad_b_noalloc(d_grad, d_off, T: int, total_elems: int, lloyd_iters: int, d_levels, d_thresh,
+                                 d_status, stream=None) -> None:
+    """BinGrad-b levels with the solver's scratch held inside the library (no workspace argument).
+
+    For callers that may not allocate device memory; at most 1024 tensors per call, and calls that
+    overlap on the GPU must be ordered because they share the one built-in scratch array."""
+    _check(
+        lib().ogq_levels_bingrad_b_noalloc(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(lloyd_iters),
+                                           _ptr(d_levels), _ptr(d_thresh), _ptr(d_status), _stream(stream)),
+        "ogq_levels_bingrad_b_noalloc",
     )
 
 

@@ -7,6 +7,8 @@
 #include "../../include/ogq.h"
 #include "ogq_internal.h"
 
+static_assert(OGQ_NOALLOC_MAX_TENSORS == ogq::kNoAllocMaxTensors, "header and library limits differ");
+
 namespace ogq {
 
 struct ProfRec {
@@ -142,6 +144,24 @@ ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, 
         e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_BINGRAD_PB, 2, d_levels, d_status,
                                       d_ws, ws_bytes, sms, (cudaStream_t)stream);
     }
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_levels_bingrad_b_noalloc(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                                        int lloyd_iters, float* d_levels, float* d_thresh,
+                                        int32_t* d_status, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_thresh || !d_status || lloyd_iters < 0 ||
+        lloyd_iters > 1024)
+        return OGQ_ERR_INVALID_ARG;
+    if (T > OGQ_NOALLOC_MAX_TENSORS) return OGQ_ERR_LIMIT;
+    if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
+    if (T == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_levels_bingrad_b_static(d_grad, d_off, T, total_elems, lloyd_iters, d_levels,
+                                                        d_thresh, d_status, sms, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return OGQ_ERR_LIMIT;
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 

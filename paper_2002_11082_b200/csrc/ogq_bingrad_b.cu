@@ -146,4 +146,52 @@ cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, i
 
 size_t ws_bytes_bingrad_b(int T, int64_t /*total*/) { return bb_ws_bytes(T, kMaxFlatCtas); }
 
+// ---------------------------------------------------------------------------
+// Variant for callers that cannot allocate device memory: the scratch of the
+// BinGrad-b solver lives in a fixed array inside the library image.  The array
+// is sized for kNoAllocMaxTensors tensors and the largest flat grid; every GPU
+// that loads the library keeps these ~304 KB until the process exits.
+// ---------------------------------------------------------------------------
+constexpr size_t kNoAllocBytes = 2 * ((sizeof(BbPart) * kMaxFlatCtas + 255) / 256 * 256) +
+                                 (sizeof(BbPart) * kNoAllocMaxTensors + 255) / 256 * 256 +
+                                 (sizeof(unsigned) * kNoAllocMaxTensors + 255) / 256 * 256 +
+                                 (sizeof(int) * kNoAllocMaxTensors + 255) / 256 * 256 +
+                                 (sizeof(long long) * kNoAllocMaxTensors + 255) / 256 * 256;
+
+static __device__ __align__(256) unsigned char g_bb_static_scratch[kNoAllocBytes];
+
+// Device address of the array above, looked up once per device.  In host code the symbol's name is
+// only a handle, not an address the GPU can use, so the address has to come from the runtime.
+static void* g_bb_static_ptr[kNoAllocMaxDevices] = {nullptr};
+
+cudaError_t launch_levels_bingrad_b_static(const float* d_grad, const int64_t* d_off, int T, int64_t total,
+                                           int lloyd_iters, float* d_levels, float* d_thresh,
+                                           int32_t* d_status, int sm_count, cudaStream_t stream)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return cudaErrorInvalidDevice;
+    if (g_bb_static_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_bb_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_bb_static_ptr[dev] = p;
+    }
+    int target = sm_count * 4 < kMaxFlatCtas ? sm_count * 4 : kMaxFlatCtas;
+    FlatGrid g = make_flat_grid(total, target, 8192);
+    if (bb_ws_bytes(T, g.ctas) > kNoAllocBytes) return cudaErrorInvalidValue;
+    BbWs ws = bb_ws_carve(g_bb_static_ptr[dev], T, g.ctas);
+    // the array still holds the previous call's counters: clear the part this call uses
+    e = cudaMemsetAsync(g_bb_static_ptr[dev], 0, bb_ws_bytes(T, g.ctas), stream);
+    if (e != cudaSuccess) return e;
+    for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
+        launch_begin("k_bb_pass", stream);
+        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters,
+                                                   d_levels, d_thresh, d_status, ws);
+        launch_end(stream);
+    }
+    return cudaGetLastError();
+}
+
 }  // namespace ogq

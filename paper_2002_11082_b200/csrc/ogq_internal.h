@@ -18,6 +18,12 @@ cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, i
                                     void* d_ws, int sm_count, cudaStream_t stream);
 size_t ws_bytes_bingrad_b(int T, int64_t total);
 
+constexpr int kNoAllocMaxTensors = 1024;  // tensors per call of the fixed-scratch BinGrad-b variant
+constexpr int kNoAllocMaxDevices = 64;
+cudaError_t launch_levels_bingrad_b_static(const float* d_grad, const int64_t* d_off, int T, int64_t total,
+                                           int lloyd_iters, float* d_levels, float* d_thresh,
+                                           int32_t* d_status, int sm_count, cudaStream_t stream);
+
 cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int T, int64_t total,
                                  int scheme, int s, float* d_levels, int32_t* d_status, void* d_ws,
                                  size_t ws_bytes, int sm_count, cudaStream_t stream);
