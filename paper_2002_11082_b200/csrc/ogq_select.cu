@@ -17,6 +17,8 @@
 // is found with one atomic counter per tensor.
 #include <math.h>
 
+#include <vector>
+
 #include "ogq_common.cuh"
 #include "ogq_internal.h"
 #include "ogq_select_solver.cuh"
@@ -33,10 +35,12 @@ constexpr int kSliceElems = 16384;
 constexpr int kMaxRounds = 32;
 constexpr int kSortScanMax = 65536;  // longest copied-key list one CTA filters for the sorting finish
 
-static_assert(2 * (256 - kSelW + (kSelW << kSelM)) <= kCells, "round-1 cells exceed the budget");
+constexpr int kRound1Mag = 256 - kSelW + (kSelW << kSelM);  // round-1 cells per sign
+constexpr int kRound1Cells = 2 * kRound1Mag;
+static_assert(kRound1Cells <= kCells, "round-1 cells exceed the budget");
 
 struct TState {
-    int done, round, m, status;
+    int done, round, m, hi_e;
     unsigned kmin_inv, kmax, nonfinite, arrive;
     unsigned expected, pad0;
     unsigned long long cursor[2];
@@ -44,7 +48,25 @@ struct TState {
     double stot;
     Interval iv[kMaxIv];
     ExactLv lv[kMaxLv];
+#ifdef OGQ_SOLVER_TIMING
+    long long tick[16];  // clock64() stamps of the last solver pass (debug builds only)
+#endif
 };
+
+#ifdef OGQ_SOLVER_TIMING
+#define OGQ_TICK(st, i) do { if (threadIdx.x == 0) (st)->tick[i] = clock64(); } while (0)
+// per-CTA wall-clock record of the round-1 and round-2 kernels: start, end, time in solver passes, passes
+__device__ unsigned long long g_dbg_cta[2][4096][4];
+__device__ __forceinline__ unsigned long long dbg_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define OGQ_CTA_BEGIN(k) unsigned long long dbg_t0 = dbg_now(), dbg_solver = 0, dbg_passes = 0; const int dbg_k = (k);
+#define OGQ_CTA_SOLVER(expr) do { unsigned long long a_ = dbg_now(); expr; dbg_solver += dbg_now() - a_; ++dbg_passes; } while (0)
+#define OGQ_CTA_END() do { if (threadIdx.x == 0 && blockIdx.x < 4096) { g_dbg_cta[dbg_k][blockIdx.x][0] = dbg_t0; g_dbg_cta[dbg_k][blockIdx.x][1] = dbg_now(); g_dbg_cta[dbg_k][blockIdx.x][2] = dbg_solver; g_dbg_cta[dbg_k][blockIdx.x][3] = dbg_passes; } } while (0)
+#else
+#define OGQ_TICK(st, i) do { } while (0)
+#define OGQ_CTA_BEGIN(k)
+#define OGQ_CTA_SOLVER(expr) do { expr; } while (0)
+#define OGQ_CTA_END() do { } while (0)
+#endif
 
 struct SelWs {
     TState* st;                  // [T]
@@ -88,7 +110,7 @@ static SelWs sel_carve(void* base, int T, int64_t total)
 // ---------------------------------------------------------------------------
 constexpr size_t kSmemHist = 3 * kCells * sizeof(uint32_t);
 constexpr size_t kSmemStage = kWarps * kStageCap * sizeof(uint32_t);
-constexpr size_t kSmemSolver = kSlots * (sizeof(uint32_t) + sizeof(double)) + 16;
+constexpr size_t kSmemSolver = kSlots * (sizeof(uint32_t) + sizeof(double) + 1) + 32;
 constexpr size_t kSmemBytes = (kSmemHist + kSmemStage > kSmemSolver) ? kSmemHist + kSmemStage : kSmemSolver;
 
 struct Table {  // interval lookup table of the tensor being streamed
@@ -97,6 +119,8 @@ struct Table {  // interval lookup table of the tensor being streamed
     int sh[kMaxIv];
     int cellbase[kMaxIv];
     int m, ncells;
+    int lo_e;                                      // bottom binade of the round-1 fine window
+    uint32_t prefilter[(kRound1Cells + 31) / 32];  // round-1 cells that touch a candidate interval
 };
 
 __device__ __forceinline__ void table_from_intervals(Table& tb, const Interval* iv, int m)
@@ -138,6 +162,41 @@ __device__ __forceinline__ int round1_intervals(int hi_e, bool magnitude_only, I
     add(0x80000000u + ((uint32_t)lo_e << 23), kSelW << kSelM, 23 - kSelM);
     add(0x80000000u + ((uint32_t)hi_e << 23), 256 - hi_e, 23);
     return m;
+}
+
+// Round-1 cell of a value, computed directly (same layout as round1_intervals produces):
+// magnitude cells ascend with |v|; negative values mirror them below, non-negative ones above.
+__device__ __forceinline__ void round1_cell(uint32_t bits, int lo_e, bool magnitude_only, int& cell,
+                                            uint32_t& lowkey)
+{
+    const uint32_t mag = bits & 0x7fffffffu;
+    const uint32_t rel = mag - ((uint32_t)lo_e << 23);
+    const int e = (int)(mag >> 23);
+    const bool fine = rel < ((uint32_t)kSelW << 23);
+    const int mi = fine ? lo_e + (int)(rel >> (23 - kSelM)) : ((e < lo_e) ? e : e - kSelW + (kSelW << kSelM));
+    const uint32_t mask = fine ? ((1u << (23 - kSelM)) - 1u) : 0x7fffffu;
+    const uint32_t low = mag & mask;
+    if (magnitude_only) { cell = mi; lowkey = low; }
+    else if (bits >> 31) { cell = kRound1Mag - 1 - mi; lowkey = mask - low; }
+    else { cell = kRound1Mag + mi; lowkey = low; }
+}
+
+__device__ __forceinline__ uint32_t key_to_bits(uint32_t k) { return (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k; }
+
+// Marks every round-1 cell that intersects one of the table's intervals (called by all threads).
+__device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
+{
+    for (int i = threadIdx.x; i < (kRound1Cells + 31) / 32; i += kThreads) tb.prefilter[i] = 0u;
+    __syncthreads();
+    if ((int)threadIdx.x < tb.m) {
+        int ca, cb;
+        uint32_t lk;
+        const uint32_t ba = key_to_bits(tb.klo[threadIdx.x]), bb = key_to_bits(tb.khi[threadIdx.x]);
+        round1_cell(magnitude_only ? (ba & 0x7fffffffu) : ba, tb.lo_e, magnitude_only, ca, lk);
+        round1_cell(magnitude_only ? (bb & 0x7fffffffu) : bb, tb.lo_e, magnitude_only, cb, lk);
+        for (int c = ca; c <= cb; ++c) atomicOr(&tb.prefilter[c >> 5], 1u << (c & 31));
+    }
+    __syncthreads();
 }
 
 __device__ __forceinline__ bool classify(const Table& tb, uint32_t key, int& cell, uint32_t& low, int& sh)
@@ -260,15 +319,21 @@ __device__ __forceinline__ void stream_piece(const void* __restrict__ src, int64
             for (int j = 0; j < 4; ++j) {
                 if (j < nv) {
                     uint32_t bits = __float_as_uint(x[j]);
-                    if (FIRST && (bits & 0x7f800000u) == 0x7f800000u) nonfinite = 1u;
-                    uint32_t key;
-                    if (magnitude_only) key = bits | 0x80000000u;
-                    else {
-                        if (bits == 0x80000000u) bits = 0u;
-                        key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+                    if (magnitude_only) bits &= 0x7fffffffu;
+                    else if (bits == 0x80000000u) bits = 0u;
+                    int cell;
+                    uint32_t low;
+                    round1_cell(bits, tb.lo_e, magnitude_only, cell, low);
+                    if (FIRST) {
+                        if ((bits & 0x7f800000u) == 0x7f800000u) nonfinite = 1u;
+                        const uint32_t key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+                        kmin = key < kmin ? key : kmin;
+                        kmax = key > kmax ? key : kmax;
+                        hist_add(cnt, lo, hi, cell, low);
+                    } else if ((tb.prefilter[cell >> 5] >> (cell & 31)) & 1u) {
+                        const uint32_t key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+                        handle(key, kk, c);
                     }
-                    if (FIRST) { kmin = key < kmin ? key : kmin; kmax = key > kmax ? key : kmax; }
-                    handle(key, kk, c);
                 }
             }
             if (COMPACT) stg.append(kk, c);
@@ -351,6 +416,8 @@ struct SolverShared {
     double ss[kWarps];
     int pb_a, pb_b, pb_c;
     int done, nm, internal;
+    uint32_t offc[kMaxIv];    // per-interval shifts of the scanned prefix arrays
+    double offs[kMaxIv];
     long long cand;           // elements inside the new intervals
     int n_keys, n_unique;     // sorting finish
     int ivstart[kMaxIv], ivufirst[kMaxIv];
@@ -503,7 +570,7 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
         int cb = 0;
         for (int j = 0; j < S.nm; ++j) { S.niv[j].sh = 0; S.niv[j].cellbase = cb; cb += S.niv[j].ncell; }
         SolverView xv;
-        xv.xkeys = xkeys; xv.cpre = xcpre; xv.spre = xspre; xv.iv = S.niv; xv.m = S.nm;
+        xv.slot_iv = nullptr; xv.xkeys = xkeys; xv.cpre = xcpre; xv.spre = xspre; xv.iv = S.niv; xv.m = S.nm;
         xv.n = S.view.n; xv.stot = S.view.stot;
         sel_init_slots(xv);
         int ra[kMaxLv], rb[kMaxLv];
@@ -528,16 +595,21 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
                              unsigned* nitems, int2* items, const uint32_t* round_buf, unsigned char* smem,
                              SolverShared& S)
 {
+    constexpr size_t kOffSpre = (kSlots * sizeof(uint32_t) + 15) / 16 * 16;
     uint32_t* cpre = reinterpret_cast<uint32_t*>(smem);
-    double* spre = reinterpret_cast<double*>(smem + ((kSlots * sizeof(uint32_t) + 15) / 16) * 16);
+    double* spre = reinterpret_cast<double*>(smem + kOffSpre);
+    uint8_t* slot_iv = smem + kOffSpre + kSlots * sizeof(double);
     const bool pb = scheme == OGQ_BINGRAD_PB;
     const int round = st->round;
+    OGQ_TICK(st, 0);
 
+    __syncthreads();
+    if ((int)threadIdx.x < st->m) S.iv[threadIdx.x] = st->iv[threadIdx.x];
     __syncthreads();
     if (threadIdx.x == 0) {
         S.view.m = st->m;
-        for (int j = 0; j < st->m; ++j) S.iv[j] = st->iv[j];
         S.view.iv = S.iv;
+        S.view.slot_iv = slot_iv;
         S.view.xkeys = nullptr;
         S.view.cpre = cpre;
         S.view.spre = spre;
@@ -548,60 +620,77 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     }
     __syncthreads();
 
-    // prefix arrays, interval by interval
-    for (int j = 0; j < S.view.m; ++j) {
-        const Interval iv = S.iv[j];
-        const int per = (iv.ncell + kThreads - 1) / kThreads;
-        const int c0 = threadIdx.x * per;
-        int c1 = c0 + per;
-        if (c1 > iv.ncell) c1 = iv.ncell;
+    // ---- prefix arrays over all slots: raw cell values, one block scan, per-interval shifts
+    const int nslots = S.view.nslots, m = S.view.m;
+    const int per = (nslots + kThreads - 1) / kThreads;
+    const int s0 = (int)threadIdx.x * per < nslots ? (int)threadIdx.x * per : nslots;
+    const int s1 = s0 + per < nslots ? s0 + per : nslots;
+    {
+        int j = 0;
+        if (s0 < nslots) {
+            int lo = 0, hi = m;
+            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (S.view.slotbase[mid] <= s0) lo = mid; else hi = mid; }
+            j = lo;
+        }
         unsigned long long lc = 0;
         double ls = 0.0;
-        for (int c = c0; c < c1; ++c) {
-            const unsigned long long cn = __ldcg(gcnt + iv.cellbase + c);
-            const unsigned long long lsum = __ldcg(glsum + iv.cellbase + c);
+        for (int slot = s0; slot < s1; ++slot) {
+            while (slot >= S.view.slotbase[j + 1]) ++j;
+            slot_iv[slot] = (uint8_t)j;
+            const int c = slot - S.view.slotbase[j];
+            unsigned long long cn = 0;
+            double sm = 0.0;
+            if (c < S.iv[j].ncell) {
+                cn = __ldcg(gcnt + S.iv[j].cellbase + c);
+                const unsigned long long lsum = __ldcg(glsum + S.iv[j].cellbase + c);
+                sm = sel_cell_sum(S.iv[j].klo + ((uint32_t)c << S.iv[j].sh), S.iv[j].sh, cn, lsum);
+            }
+            cpre[slot] = (uint32_t)cn;
+            spre[slot] = sm;
             lc += cn;
-            ls += sel_cell_sum(iv.klo + ((uint32_t)c << iv.sh), iv.sh, cn, lsum);
+            ls += sm;
         }
         unsigned long long tc;
         double ts;
         block_excl_scan(lc, ls, S.sc, S.ss, tc, ts);
-        unsigned long long bc = (unsigned long long)iv.cbefore;
-        double bs = iv.sbefore;
-        if (round == 1 && j > 0) {  // round-1 intervals tile the key line: chain them
-            bc = cpre[S.view.slotbase[j] - 1];
-            bs = spre[S.view.slotbase[j] - 1];
+        for (int slot = s0; slot < s1; ++slot) {
+            const unsigned long long cn = cpre[slot];
+            const double sm = spre[slot];
+            cpre[slot] = (uint32_t)lc;
+            spre[slot] = ls;
+            lc += cn;
+            ls += sm;
         }
-        unsigned long long rc = bc + lc;
-        double rs = bs + ls;
-        const int sb = S.view.slotbase[j];
-        for (int c = c0; c < c1; ++c) {
-            cpre[sb + c] = (uint32_t)rc;
-            spre[sb + c] = rs;
-            const unsigned long long cn = __ldcg(gcnt + iv.cellbase + c);
-            const unsigned long long lsum = __ldcg(glsum + iv.cellbase + c);
-            rc += cn;
-            rs += sel_cell_sum(iv.klo + ((uint32_t)c << iv.sh), iv.sh, cn, lsum);
-        }
-        if (threadIdx.x == 0) {
-            cpre[sb + iv.ncell] = (uint32_t)(bc + tc);
-            spre[sb + iv.ncell] = bs + ts;
-            if (round == 1) { S.iv[j].cbefore = (long long)bc; S.iv[j].sbefore = bs; }
-        }
-        __syncthreads();
-    }
-    if (threadIdx.x == 0 && round == 1) {
-        st->stot = spre[S.view.nslots - 1];
-        if ((long long)cpre[S.view.nslots - 1] != st->n) S.internal = 1;
     }
     __syncthreads();
-    if (threadIdx.x == 0) S.view.stot = st->stot;
+    if ((int)threadIdx.x < m) {
+        // rounds >= 2: shift every interval so that it starts from the exact (count, sum) before it
+        const int sb = S.view.slotbase[threadIdx.x];
+        S.offc[threadIdx.x] = (round == 1) ? 0u : (uint32_t)((unsigned long long)S.iv[threadIdx.x].cbefore - cpre[sb]);
+        S.offs[threadIdx.x] = (round == 1) ? 0.0 : S.iv[threadIdx.x].sbefore - spre[sb];
+    }
     __syncthreads();
+    if (round != 1)
+        for (int slot = s0; slot < s1; ++slot) {
+            const int j = slot_iv[slot];
+            cpre[slot] += S.offc[j];
+            spre[slot] += S.offs[j];
+        }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (round == 1) {
+            st->stot = spre[nslots - 1];
+            if ((long long)cpre[nslots - 1] != st->n) S.internal = 1;
+        }
+        S.view.stot = st->stot;
+    }
+    __syncthreads();
+    OGQ_TICK(st, 1);
 
     if (pb && !S.internal && S.view.stot > 0.0) {
         // bracket of the sign change of g, evaluated at the lower edge of every cell
         int a = -1, b = -1, cs = -1;
-        for (int sl = threadIdx.x; sl < S.view.nslots; sl += kThreads) {
+        for (int sl = threadIdx.x; sl < nslots; sl += kThreads) {
             if (sel_is_end_slot(S.view, sl)) continue;
             double x;
             const double g = sel_pb_g(S.view, sl, &x);
@@ -615,7 +704,35 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         if (b >= 0) atomicMax(&S.pb_b, b);
         if (cs >= 0) atomicMax(&S.pb_c, cs);
     }
+    if (!pb && !S.internal) {
+        // one thread per level, one depth of Algorithm 1 at a time
+        if ((int)threadIdx.x < s) {
+            LvInfo& l = S.lv[threadIdx.x];
+            if (round == 1) {
+                l.exact = 0;
+                if (threadIdx.x == 0) {
+                    l.exact = 1; l.key = ~__ldcg(&st->kmin_inv); l.val = (double)sel_key_to_float(l.key);
+                    l.c_lt = 0; l.s_lt = 0.0; l.c_le = 0; l.s_le = 0.0;
+                } else if ((int)threadIdx.x == s - 1) {
+                    l.exact = 1; l.key = __ldcg(&st->kmax); l.val = (double)sel_key_to_float(l.key);
+                    l.c_lt = 0; l.s_lt = 0.0; l.c_le = S.view.n; l.s_le = S.view.stot;
+                }
+            } else {
+                const ExactLv& e = st->lv[threadIdx.x];
+                l.exact = e.exact; l.key = e.key; l.val = (double)sel_key_to_float(e.key);
+                l.c_lt = e.c_lt; l.c_le = e.c_le; l.s_lt = e.s_lt; l.s_le = e.s_le;
+            }
+        }
+        for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
+            __syncthreads();
+            const int q = threadIdx.x;
+            if (q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0 && !S.lv[q].exact) {
+                if (!sel_orq_solve(S.view, S.lv[q - stride], S.lv[q + stride], S.lv[q])) S.internal = 1;
+            }
+        }
+    }
     __syncthreads();
+    OGQ_TICK(st, 2);
 
     if (threadIdx.x == 0) {
         int ra[kMaxLv], rb[kMaxLv];
@@ -646,28 +763,9 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
                 }
             }
         } else {
-            if (round == 1) {
-                for (int q = 0; q < s; ++q) S.lv[q].exact = 0;
-                LvInfo& l0 = S.lv[0];
-                l0.exact = 1; l0.key = ~__ldcg(&st->kmin_inv); l0.val = (double)sel_key_to_float(l0.key);
-                l0.c_lt = 0; l0.s_lt = 0.0; l0.c_le = 0; l0.s_le = 0.0;
-                LvInfo& l1 = S.lv[s - 1];
-                l1.exact = 1; l1.key = __ldcg(&st->kmax); l1.val = (double)sel_key_to_float(l1.key);
-                l1.c_lt = 0; l1.s_lt = 0.0; l1.c_le = st->n; l1.s_le = st->stot;
-            } else {
-                for (int q = 0; q < s; ++q) {
-                    const ExactLv& e = st->lv[q];
-                    S.lv[q].exact = e.exact;
-                    S.lv[q].key = e.key;
-                    S.lv[q].val = (double)sel_key_to_float(e.key);
-                    S.lv[q].c_lt = e.c_lt; S.lv[q].c_le = e.c_le; S.lv[q].s_lt = e.s_lt; S.lv[q].s_le = e.s_le;
-                }
-            }
-            open = sel_orq_pass(S.view, s, S.lv, ra, rb);
-            if (open < 0) {
-                stbits = OGQ_ST_INTERNAL;
-                S.done = 1;
-            } else if (open == 0) {
+            for (int q = 1; q < s - 1; ++q)
+                if (!S.lv[q].exact) { ra[open] = S.lv[q].sa; rb[open] = S.lv[q].sb; ++open; }
+            if (open == 0) {
                 for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = sel_key_to_float(S.lv[q].key);
                 S.done = 1;
             } else {
@@ -694,17 +792,21 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
             else for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
         }
         if (stbits) status[t] |= stbits;
+        OGQ_TICK(st, 3);
     }
     __syncthreads();
 
     if (S.done) {
         if (threadIdx.x == 0) { st->done = 1; __threadfence(); }
+        OGQ_TICK(st, 5);
         return true;
     }
     if (!pb && round >= 2 && S.cand <= kSmallN && round_buf != nullptr) {
         const long long src_cnt = (long long)__ldcg(&st->cursor[round & 1]);
         if (src_cnt <= kSortScanMax) {
+            OGQ_TICK(st, 4);
             sort_finish(st, t, s, round_buf, src_cnt, levels, status, smem, S);
+            OGQ_TICK(st, 5);
             return true;
         }
     }
@@ -714,8 +816,8 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         gcnt[i] = 0u;
         glsum[i] = 0ull;
     }
+    if ((int)threadIdx.x < S.nm) st->iv[threadIdx.x] = S.niv[threadIdx.x];
     if (threadIdx.x == 0) {
-        for (int j = 0; j < S.nm; ++j) st->iv[j] = S.niv[j];
         st->m = S.nm;
         st->round = round + 1;
         st->arrive = 0;
@@ -733,6 +835,7 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     }
     __threadfence();
     __syncthreads();
+    OGQ_TICK(st, 5);
     return false;
 }
 
@@ -966,6 +1069,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
     const int64_t lo = (int64_t)blockIdx.x * A.chunk;
     const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
+    OGQ_CTA_BEGIN(0)
 
     for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
         const int64_t n = tend - tbeg;
@@ -991,6 +1095,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
             if (hi_e > 256) hi_e = 256;
             const int m = round1_intervals(hi_e, pb, r1iv);
             table_from_intervals(tb, r1iv, m);
+            tb.lo_e = hi_e - kSelW;
         }
         __syncthreads();
         zero_hist(hist, tb.ncells);
@@ -1036,6 +1141,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
         if (threadIdx.x == 0) {
             st->n = n;
             st->round = 1;
+            st->hi_e = tb.lo_e + kSelW;
             st->m = tb.m;
             for (int j = 0; j < tb.m; ++j) st->iv[j] = r1iv[j];
             int stb = 0;
@@ -1055,9 +1161,10 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
         }
         __syncthreads();
         if (sh_last & (OGQ_ST_NONFINITE | OGQ_ST_CONSTANT)) return;
-        solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                     A.levels, A.status, A.ws.nitems, A.ws.items, nullptr, smem, S);
+        OGQ_CTA_SOLVER(solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme,
+                                    A.s, A.levels, A.status, A.ws.nitems, A.ws.items, nullptr, smem, S));
     });
+    OGQ_CTA_END();
 }
 
 __global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
@@ -1070,6 +1177,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
     const int64_t lo = (int64_t)blockIdx.x * A.chunk;
     const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
+    OGQ_CTA_BEGIN(1)
 
     for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
         const int64_t n = tend - tbeg;
@@ -1077,8 +1185,12 @@ __global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
         TState* st = A.ws.st + t;
         if (__ldcg(&st->done)) return;
         __syncthreads();
-        if (threadIdx.x == 0) table_from_intervals(tb, st->iv, __ldcg(&st->m));
+        if (threadIdx.x == 0) {
+            table_from_intervals(tb, st->iv, __ldcg(&st->m));
+            tb.lo_e = st->hi_e - kSelW;
+        }
         __syncthreads();
+        build_prefilter(tb, pb);
         zero_hist(hist, tb.ncells);
         __syncthreads();
         Stager stg;
@@ -1102,9 +1214,10 @@ __global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
         __syncthreads();
         if (!sh_last) return;
         __threadfence();
-        solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                     A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, smem, S);
+        OGQ_CTA_SOLVER(solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme,
+                                    A.s, A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, smem, S));
     });
+    OGQ_CTA_END();
 }
 
 __global__ void __launch_bounds__(kThreads) k_sel_round3(SelArgs A)
@@ -1158,6 +1271,24 @@ __global__ void __launch_bounds__(kThreads) k_sel_round3(SelArgs A)
             finish_alone(A, t, smem, tb, S);
     }
 }
+
+#ifdef OGQ_SOLVER_TIMING
+extern "C" int ogq_debug_dump_ctas(unsigned long long* h_out /*[2][4096][4]*/)
+{
+    return cudaMemcpyFromSymbol(h_out, g_dbg_cta, sizeof(unsigned long long) * 2 * 4096 * 4) == cudaSuccess ? 0 : -1;
+}
+extern "C" int ogq_debug_dump_ticks(const void* d_ws, int T, long long* h_out /*[T][16]*/, int* h_round, long long* h_n)
+{
+    std::vector<TState> h(T);
+    if (cudaMemcpy(h.data(), d_ws, sizeof(TState) * (size_t)T, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    for (int t = 0; t < T; ++t) {
+        for (int i = 0; i < 16; ++i) h_out[t * 16 + i] = h[t].tick[i];
+        h_round[t] = h[t].round;
+        h_n[t] = h[t].n;
+    }
+    return 0;
+}
+#endif
 
 cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int T, int64_t total, int scheme,
                                  int s, float* d_levels, int32_t* d_status, void* d_ws, size_t /*ws_bytes*/,

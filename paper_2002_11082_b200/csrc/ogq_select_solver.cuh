@@ -83,14 +83,21 @@ OGQ_HD double sel_cell_sum(uint32_t kbase, int sh, unsigned long long cnt, unsig
         sign = -1.0;
     }
     const int e = (int)(mag0 >> 23);
-    if (e == 0) return sign * ldexp((double)magsum, -149);
-    const unsigned long long mant = magsum - cnt * ((unsigned long long)(e - 1) << 23);
-    return sign * ldexp((double)mant, e - 150);
+    // value = mant * 2^(max(e,1) - 150); for e = 0 (subnormals) mant is the plain sum of magnitudes
+    const unsigned long long mant = (e == 0) ? magsum : magsum - cnt * ((unsigned long long)(e - 1) << 23);
+    const int ee = (e == 0) ? 1 : e;
+#ifdef __CUDA_ARCH__
+    const double scale = __hiloint2double((ee + 873) << 20, 0);  // 2^(ee - 150), exact
+    return sign * (__ull2double_rn(mant) * scale);
+#else
+    return sign * ldexp((double)mant, ee - 150);
+#endif
 }
 
 // Prefix arrays over "slots": interval j owns slots [slotbase[j], slotbase[j] + ncell_j]; slot
 // slotbase[j] + c is the state before its cell c, the last one the state after its last cell.
 struct SolverView {
+    const uint8_t* slot_iv;  // optional: interval index of every slot (null: searched)
     const uint32_t* xkeys;  // explicit mode: cell c of the view holds the single key xkeys[c] (else null)
     const uint32_t* cpre;  // #{elements before the slot} (absolute)
     const double* spre;    // their sum
@@ -115,9 +122,13 @@ OGQ_HD void sel_init_slots(SolverView& v)
 
 OGQ_HD int sel_interval_of_slot(const SolverView& v, int slot)
 {
-    int j = 0;
-    while (j + 1 < v.m && v.slotbase[j + 1] <= slot) ++j;
-    return j;
+    if (v.slot_iv) return v.slot_iv[slot];
+    int lo = 0, hi = v.m;  // last interval whose first slot is <= slot
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (v.slotbase[mid] <= slot) lo = mid; else hi = mid;
+    }
+    return lo;
 }
 
 OGQ_HD bool sel_is_end_slot(const SolverView& v, int slot)
