@@ -26,10 +26,13 @@
 
 namespace ogq {
 
+constexpr int kSelThreads = 1024;   // one CTA per SM; 32 warps keep enough loads in flight
+constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelW = 16;          // binades in the fine window of round 1
 constexpr int kSelM = 7;           // log2(cells per binade) in the window
 constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
-constexpr int kStageCap = 512;     // per-warp staging entries for compaction
+constexpr int kMidN = 131072;      // tensors up to this size are solved start to finish by one CTA of their own
+constexpr int kStageCap = 256;     // per-warp staging entries for compaction
 constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
 constexpr int kSliceElems = 16384;
 constexpr int kMaxRounds = 32;
@@ -109,7 +112,7 @@ static SelWs sel_carve(void* base, int T, int64_t total)
 // solver reuses the same bytes for its prefix arrays.
 // ---------------------------------------------------------------------------
 constexpr size_t kSmemHist = 3 * kCells * sizeof(uint32_t);
-constexpr size_t kSmemStage = kWarps * kStageCap * sizeof(uint32_t);
+constexpr size_t kSmemStage = kSelWarps * kStageCap * sizeof(uint32_t);
 constexpr size_t kSmemSolver = kSlots * (sizeof(uint32_t) + sizeof(double) + 1) + 32;
 constexpr size_t kSmemBytes = (kSmemHist + kSmemStage > kSmemSolver) ? kSmemHist + kSmemStage : kSmemSolver;
 
@@ -186,7 +189,7 @@ __device__ __forceinline__ uint32_t key_to_bits(uint32_t k) { return (k & 0x8000
 // Marks every round-1 cell that intersects one of the table's intervals (called by all threads).
 __device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
 {
-    for (int i = threadIdx.x; i < (kRound1Cells + 31) / 32; i += kThreads) tb.prefilter[i] = 0u;
+    for (int i = threadIdx.x; i < (kRound1Cells + 31) / 32; i += kSelThreads) tb.prefilter[i] = 0u;
     __syncthreads();
     if ((int)threadIdx.x < tb.m) {
         int ca, cb;
@@ -245,14 +248,22 @@ __device__ __forceinline__ void warp_visit4(const E* __restrict__ base, int64_t 
     }
     const E4* b4 = reinterpret_cast<const E4*>(base);
     const int64_t e = b >> 2;
-    for (int64_t i0 = (a >> 2) + warp * 32; i0 < e; i0 += 2 * kThreads) {
-        const int64_t i = i0 + lane, i2 = i + kThreads;
-        E x[4], y[4];
-        int nx = 0, ny = 0;
-        if (i < e) { const E4 v = ld4(b4 + i); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; nx = 4; }
-        if (i2 < e) { const E4 v = ld4(b4 + i2); y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w; ny = 4; }
-        f(x, nx);
-        if (i0 + kThreads < e) f(y, ny);
+    for (int64_t i0 = (a >> 2) + warp * 32; i0 < e; i0 += 4 * kSelThreads) {
+        E x[4][4];
+        int nx[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t i = i0 + (int64_t)u * kSelThreads + lane;
+            nx[u] = 0;
+            if (i < e) {
+                const E4 v = ld4(b4 + i);
+                x[u][0] = v.x; x[u][1] = v.y; x[u][2] = v.z; x[u][3] = v.w;
+                nx[u] = 4;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i0 + (int64_t)u * kSelThreads < e) f(x[u], nx[u]);
     }
 }
 
@@ -352,7 +363,7 @@ __device__ __forceinline__ void stream_piece(const void* __restrict__ src, int64
 
 __device__ __forceinline__ void zero_hist(uint32_t* smem_hist, int ncells)
 {
-    for (int i = threadIdx.x; i < ncells; i += kThreads) {
+    for (int i = threadIdx.x; i < ncells; i += kSelThreads) {
         smem_hist[i] = 0u;
         smem_hist[kCells + i] = 0u;
         smem_hist[2 * kCells + i] = 0u;
@@ -362,7 +373,7 @@ __device__ __forceinline__ void zero_hist(uint32_t* smem_hist, int ncells)
 __device__ __forceinline__ void flush_hist(const uint32_t* smem_hist, int ncells, uint32_t* gcnt,
                                            unsigned long long* glsum)
 {
-    for (int i = threadIdx.x; i < ncells; i += kThreads) {
+    for (int i = threadIdx.x; i < ncells; i += kSelThreads) {
         const uint32_t c = smem_hist[i];
         if (c) {
             atomicAdd(gcnt + i, c);
@@ -371,6 +382,20 @@ __device__ __forceinline__ void flush_hist(const uint32_t* smem_hist, int ncells
             if (l) atomicAdd(glsum + i, l);
         }
     }
+}
+
+// Sum of a double over the CTA in a fixed order; valid in thread 0.  scratch: kSelWarps doubles.
+__device__ __forceinline__ double sel_block_sum(double x, double* scratch)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = x;
+    __syncthreads();
+    double r = 0.0;
+    if (threadIdx.x == 0)
+        for (int i = 0; i < kSelWarps; ++i) r += scratch[i];
+    return r;
 }
 
 // ---------------------------------------------------------------------------
@@ -398,7 +423,7 @@ __device__ __forceinline__ void block_excl_scan(unsigned long long& c, double& s
     tot_c = 0;
     tot_s = 0.0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < kSelWarps; ++w) {
         if (w < warp) { bc += sc[w]; bs += ss[w]; }
         tot_c += sc[w];
         tot_s += ss[w];
@@ -412,8 +437,8 @@ struct SolverShared {
     Interval niv[kMaxIv];
     LvInfo lv[kMaxLv];
     SolverView view;
-    unsigned long long sc[kWarps];
-    double ss[kWarps];
+    unsigned long long sc[kSelWarps];
+    double ss[kSelWarps];
     int pb_a, pb_b, pb_c;
     int done, nm, internal;
     uint32_t offc[kMaxIv];    // per-interval shifts of the scanned prefix arrays
@@ -441,7 +466,7 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
                             float* __restrict__ levels, int32_t* __restrict__ status, unsigned char* smem,
                             SolverShared& S)
 {
-    constexpr int kPer = kSmallN / kThreads;
+    constexpr int kPer = kSmallN / kSelThreads;
     uint32_t* skeys = reinterpret_cast<uint32_t*>(smem);
     uint32_t* xkeys = skeys + kSmallN;
     uint32_t* xcpre = xkeys + kSmallN;
@@ -450,7 +475,7 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     if (threadIdx.x == 0) S.n_keys = 0;
     if (threadIdx.x < kMaxIv) { S.ivstart[threadIdx.x] = 0; S.ivufirst[threadIdx.x] = -1; S.ivpre[threadIdx.x] = 0.0; }
     __syncthreads();
-    for (long long i = threadIdx.x; i < src_cnt; i += kThreads) {
+    for (long long i = threadIdx.x; i < src_cnt; i += kSelThreads) {
         const uint32_t key = __ldcg(buf + i);
         if (find_new_interval(S, key) >= 0) {
             const int pos = atomicAdd(&S.n_keys, 1);
@@ -461,11 +486,11 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     const int c = S.n_keys < kSmallN ? S.n_keys : kSmallN;
     int P = 1;
     while (P < c) P <<= 1;
-    for (int i = c + threadIdx.x; i < kSmallN; i += kThreads) skeys[i] = 0xffffffffu;
+    for (int i = c + threadIdx.x; i < kSmallN; i += kSelThreads) skeys[i] = 0xffffffffu;
     __syncthreads();
     for (int k = 2; k <= P; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < P; i += kThreads) {
+            for (int i = threadIdx.x; i < P; i += kSelThreads) {
                 const int ixj = i ^ j;
                 if (ixj > i) {
                     const uint32_t a = skeys[i], b = skeys[ixj];
@@ -592,8 +617,8 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
 // Called by every thread of the CTA; returns true when the tensor is finished.
 __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long long* glsum, int scheme,
                              int s, float* __restrict__ levels, int32_t* __restrict__ status,
-                             unsigned* nitems, int2* items, const uint32_t* round_buf, unsigned char* smem,
-                             SolverShared& S)
+                             unsigned* nitems, int2* items, const uint32_t* round_buf, bool enqueue,
+                             unsigned char* smem, SolverShared& S)
 {
     constexpr size_t kOffSpre = (kSlots * sizeof(uint32_t) + 15) / 16 * 16;
     uint32_t* cpre = reinterpret_cast<uint32_t*>(smem);
@@ -622,34 +647,42 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
 
     // ---- prefix arrays over all slots: raw cell values, one block scan, per-interval shifts
     const int nslots = S.view.nslots, m = S.view.m;
-    const int per = (nslots + kThreads - 1) / kThreads;
+    const int per = (nslots + kSelThreads - 1) / kSelThreads;
     const int s0 = (int)threadIdx.x * per < nslots ? (int)threadIdx.x * per : nslots;
     const int s1 = s0 + per < nslots ? s0 + per : nslots;
     {
+        // interval index of every slot (blocked over threads, no global traffic)
         int j = 0;
         if (s0 < nslots) {
             int lo = 0, hi = m;
             while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (S.view.slotbase[mid] <= s0) lo = mid; else hi = mid; }
             j = lo;
         }
-        unsigned long long lc = 0;
-        double ls = 0.0;
         for (int slot = s0; slot < s1; ++slot) {
             while (slot >= S.view.slotbase[j + 1]) ++j;
             slot_iv[slot] = (uint8_t)j;
-            const int c = slot - S.view.slotbase[j];
+        }
+        __syncthreads();
+        // raw (count, sum) of every cell: strided so that the global loads are coalesced and independent
+#pragma unroll 4
+        for (int slot = threadIdx.x; slot < nslots; slot += kSelThreads) {
+            const int jj = slot_iv[slot];
+            const int c = slot - S.view.slotbase[jj];
             unsigned long long cn = 0;
             double sm = 0.0;
-            if (c < S.iv[j].ncell) {
-                cn = __ldcg(gcnt + S.iv[j].cellbase + c);
-                const unsigned long long lsum = __ldcg(glsum + S.iv[j].cellbase + c);
-                sm = sel_cell_sum(S.iv[j].klo + ((uint32_t)c << S.iv[j].sh), S.iv[j].sh, cn, lsum);
+            if (c < S.iv[jj].ncell) {
+                cn = __ldcg(gcnt + S.iv[jj].cellbase + c);
+                const unsigned long long lsum = __ldcg(glsum + S.iv[jj].cellbase + c);
+                sm = sel_cell_sum(S.iv[jj].klo + ((uint32_t)c << S.iv[jj].sh), S.iv[jj].sh, cn, lsum);
             }
             cpre[slot] = (uint32_t)cn;
             spre[slot] = sm;
-            lc += cn;
-            ls += sm;
         }
+        __syncthreads();
+        // exclusive prefix: per-thread blocks, one block scan, in place
+        unsigned long long lc = 0;
+        double ls = 0.0;
+        for (int slot = s0; slot < s1; ++slot) { lc += cpre[slot]; ls += spre[slot]; }
         unsigned long long tc;
         double ts;
         block_excl_scan(lc, ls, S.sc, S.ss, tc, ts);
@@ -690,7 +723,7 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     if (pb && !S.internal && S.view.stot > 0.0) {
         // bracket of the sign change of g, evaluated at the lower edge of every cell
         int a = -1, b = -1, cs = -1;
-        for (int sl = threadIdx.x; sl < nslots; sl += kThreads) {
+        for (int sl = threadIdx.x; sl < nslots; sl += kSelThreads) {
             if (sel_is_end_slot(S.view, sl)) continue;
             double x;
             const double g = sel_pb_g(S.view, sl, &x);
@@ -812,7 +845,7 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     }
     // prepare the next round: clear the cells it will use, publish the new intervals
     const int ncells_next = S.niv[S.nm - 1].cellbase + S.niv[S.nm - 1].ncell;
-    for (int i = threadIdx.x; i < ncells_next; i += kThreads) {
+    for (int i = threadIdx.x; i < ncells_next; i += kSelThreads) {
         gcnt[i] = 0u;
         glsum[i] = 0ull;
     }
@@ -823,7 +856,7 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         st->arrive = 0;
         const int next = round + 1;
         st->cursor[next & 1] = 0ull;  // buffer the next round writes
-        if (next == 3) {
+        if (next == 3 && enqueue) {
             const unsigned long long cntk = __ldcg(&st->cursor[0]);
             unsigned ns = (unsigned)((cntk + kSliceElems - 1) / kSliceElems);
             if (ns < 1) ns = 1;
@@ -860,7 +893,7 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
                              float* __restrict__ levels, int32_t* __restrict__ status, TState* st,
                              unsigned char* smem)
 {
-    __shared__ double sh_d[kWarps];
+    __shared__ double sh_d[kSelWarps];
     __shared__ uint32_t sh_lvkey[kMaxLv];
     __shared__ int sh_flag;
     __shared__ double sh_bcast;
@@ -870,7 +903,7 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
     while (P < n) P <<= 1;
     if (threadIdx.x == 0) sh_flag = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < P; i += kThreads) {
+    for (int i = threadIdx.x; i < P; i += kSelThreads) {
         uint32_t key = 0xffffffffu;
         if (i < n) {
             uint32_t bits = __float_as_uint(__ldg(grad + tb + i));
@@ -887,7 +920,7 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
     // bitonic sort, ascending
     for (int k = 2; k <= P; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < P; i += kThreads) {
+            for (int i = threadIdx.x; i < P; i += kSelThreads) {
                 const int ixj = i ^ j;
                 if (ixj > i) {
                     const uint32_t a = keys[i], b = keys[ixj];
@@ -923,8 +956,8 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
                     const int i0 = lower_bound_u32(keys, n, kl), i1 = upper_bound_u32(keys, n, kr);
                     const double Lv = (double)sel_key_to_float(kl), Rv = (double)sel_key_to_float(kr);
                     double a = 0.0;
-                    for (int i = i0 + threadIdx.x; i < i1; i += kThreads) a += (double)sel_key_to_float(keys[i]) - Lv;
-                    a = block_sum(a, sh_d);
+                    for (int i = i0 + threadIdx.x; i < i1; i += kSelThreads) a += (double)sel_key_to_float(keys[i]) - Lv;
+                    a = sel_block_sum(a, sh_d);
                     if (threadIdx.x == 0) sh_bcast = a;
                     __syncthreads();
                     a = sh_bcast;
@@ -946,10 +979,10 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
     }
     // BinGrad-pb: prefix sums of the sorted magnitudes, then the sign change of g
     double* pre = reinterpret_cast<double*>(smem + kSmallN * sizeof(uint32_t));  // [n + 1]
-    __shared__ unsigned long long sc_[kWarps];
-    __shared__ double ss_[kWarps];
+    __shared__ unsigned long long sc_[kSelWarps];
+    __shared__ double ss_[kSelWarps];
     __shared__ int sh_c;
-    const int per = (n + kThreads - 1) / kThreads;
+    const int per = (n + kSelThreads - 1) / kSelThreads;
     const int c0 = threadIdx.x * per < n ? threadIdx.x * per : n;
     const int c1 = c0 + per < n ? c0 + per : n;
     unsigned long long dummy = 0, dt;
@@ -961,7 +994,7 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
     if (threadIdx.x == 0) { pre[n] = tot; sh_c = -1; }
     __syncthreads();
     int best = -1;
-    for (int i = threadIdx.x; i < n; i += kThreads) {
+    for (int i = threadIdx.x; i < n; i += kSelThreads) {
         const double x = (double)sel_key_to_float(keys[i]);
         const int first = lower_bound_u32(keys, n, keys[i]);
         const double g = x * (double)n - (tot - pre[first]);
@@ -1031,7 +1064,7 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
         __threadfence();
         __syncthreads();
         if (solver_round(st, t, gcnt, glsum, A.scheme, A.s, A.levels, A.status, A.ws.nitems, A.ws.items,
-                         A.ws.buf[round & 1] + tbeg, smem, S))
+                         A.ws.buf[round & 1] + tbeg, false, smem, S))
             return;
     }
     if (threadIdx.x == 0) {
@@ -1040,45 +1073,30 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
     }
 }
 
-__global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
+__global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ Table tb;
     __shared__ SolverShared S;
     __shared__ Interval r1iv[kMaxIv];
-    __shared__ int sh_i[kWarps];
-    __shared__ uint32_t sh_u[2 * kWarps];
+    __shared__ int sh_i[kSelWarps];
+    __shared__ uint32_t sh_u[2 * kSelWarps];
     __shared__ int sh_last;
     const bool pb = A.scheme == OGQ_BINGRAD_PB;
     const int nl = pb ? 2 : A.s;
 
-    if ((int)blockIdx.x >= A.flat_ctas) {
-        // one extra CTA per tensor: empty and small tensors are settled here
-        const int t = blockIdx.x - A.flat_ctas;
-        const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
-        const int64_t n = tend - tbeg;
-        if (n <= 0) {
-            if (threadIdx.x < nl) A.levels[(int64_t)t * nl + threadIdx.x] = 0.f;
-            if (threadIdx.x == 0) { A.status[t] = OGQ_ST_EMPTY; A.ws.st[t].done = 1; }
-        } else if (n <= kSmallN) {
-            small_tensor(A.grad, tbeg, (int)n, t, A.scheme, A.s, A.levels, A.status, A.ws.st + t, smem);
-        }
-        return;
-    }
-
-    const int64_t lo = (int64_t)blockIdx.x * A.chunk;
-    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
     OGQ_CTA_BEGIN(0)
 
-    for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+    // Round 1 over one piece [pb_, pe_) of tensor t.  `alone`: the piece is the whole tensor and
+    // this CTA runs all of its rounds.  Returns true when the tensor is finished.
+    auto do_round1 = [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_, bool alone) -> bool {
         const int64_t n = tend - tbeg;
-        if (n <= kSmallN) return;
         TState* st = A.ws.st + t;
-        // anchor of the fine window: largest binade among 256 strided samples, plus two
+        // anchor of the fine window: largest binade among strided samples, plus two
         int e = 0;
         {
-            const int64_t idx = tbeg + (int64_t)threadIdx.x * n / kThreads;
+            const int64_t idx = tbeg + (int64_t)threadIdx.x * n / kSelThreads;
             e = (int)((__float_as_uint(__ldg(A.grad + idx)) >> 23) & 255u);
             if (e == 255) e = 0;
 #pragma unroll
@@ -1089,7 +1107,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
         __syncthreads();
         if (threadIdx.x == 0) {
             int mx = 0;
-            for (int w = 0; w < kWarps; ++w) mx = sh_i[w] > mx ? sh_i[w] : mx;
+            for (int w = 0; w < kSelWarps; ++w) mx = sh_i[w] > mx ? sh_i[w] : mx;
             int hi_e = mx + 2;
             if (hi_e < kSelW) hi_e = kSelW;
             if (hi_e > 256) hi_e = 256;
@@ -1116,28 +1134,31 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
         __syncthreads();
         if ((threadIdx.x & 31) == 0) {
             sh_u[threadIdx.x >> 5] = kmin;
-            sh_u[kWarps + (threadIdx.x >> 5)] = kmax;
+            sh_u[kSelWarps + (threadIdx.x >> 5)] = kmax;
             if (nf) atomicOr(&st->nonfinite, 1u);
         }
         __syncthreads();
         flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         if (threadIdx.x == 0) {
             uint32_t mn = 0xffffffffu, mx = 0u;
-            for (int w = 0; w < kWarps; ++w) { mn = sh_u[w] < mn ? sh_u[w] : mn; mx = sh_u[kWarps + w] > mx ? sh_u[kWarps + w] : mx; }
+            for (int w = 0; w < kSelWarps; ++w) { mn = sh_u[w] < mn ? sh_u[w] : mn; mx = sh_u[kSelWarps + w] > mx ? sh_u[kSelWarps + w] : mx; }
             atomicMax(&st->kmin_inv, ~mn);
             atomicMax(&st->kmax, mx);
         }
         __threadfence();
         __syncthreads();
-        const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
-        if (threadIdx.x == 0) {
-            const unsigned prev = atomicAdd(&st->arrive, 1u);
-            sh_last = (prev == (unsigned)(c1 - c0));
+        if (!alone) {
+            const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
+            if (threadIdx.x == 0) {
+                const unsigned prev = atomicAdd(&st->arrive, 1u);
+                sh_last = (prev == (unsigned)(c1 - c0));
+            }
+            __syncthreads();
+            if (!sh_last) return false;
+            __threadfence();
         }
-        __syncthreads();
-        if (!sh_last) return;
-        __threadfence();
         // last CTA of this tensor: set up the state and run the first solver pass
+        __syncthreads();
         if (threadIdx.x == 0) {
             st->n = n;
             st->round = 1;
@@ -1160,14 +1181,69 @@ __global__ void __launch_bounds__(kThreads) k_sel_round1(SelArgs A)
             }
         }
         __syncthreads();
-        if (sh_last & (OGQ_ST_NONFINITE | OGQ_ST_CONSTANT)) return;
-        OGQ_CTA_SOLVER(solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme,
-                                    A.s, A.levels, A.status, A.ws.nitems, A.ws.items, nullptr, smem, S));
+        if (sh_last & (OGQ_ST_NONFINITE | OGQ_ST_CONSTANT)) return true;
+        bool done;
+        OGQ_CTA_SOLVER(done = solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells,
+                                           A.scheme, A.s, A.levels, A.status, A.ws.nitems, A.ws.items, nullptr,
+                                           !alone, smem, S));
+        return done;
+    };
+
+    if ((int)blockIdx.x < A.T) {
+        // the first T CTAs, one per tensor, settle the empty, small and mid-size tensors; they come
+        // first in the grid because the mid-size ones run longest
+        const int t = blockIdx.x;
+        const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
+        const int64_t n = tend - tbeg;
+        if (n <= 0) {
+            if (threadIdx.x < nl) A.levels[(int64_t)t * nl + threadIdx.x] = 0.f;
+            if (threadIdx.x == 0) { A.status[t] = OGQ_ST_EMPTY; A.ws.st[t].done = 1; }
+        } else if (n <= kSmallN) {
+            small_tensor(A.grad, tbeg, (int)n, t, A.scheme, A.s, A.levels, A.status, A.ws.st + t, smem);
+        } else if (n <= kMidN) {
+            // all rounds on this CTA: round 1 and 2 read the tensor (it stays in L2), later rounds the copied keys
+            if (do_round1(t, tbeg, tend, tbeg, tend, true)) return;
+            TState* st = A.ws.st + t;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                table_from_intervals(tb, st->iv, st->m);
+                tb.lo_e = st->hi_e - kSelW;
+            }
+            __syncthreads();
+            build_prefilter(tb, pb);
+            zero_hist(hist, tb.ncells);
+            __syncthreads();
+            Stager stg;
+            stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+            stg.dst = A.ws.buf[0] + tbeg;
+            stg.cursor = &st->cursor[0];
+            stg.fill = 0;
+            uint32_t kmin = 0, kmax = 0, nf = 0;
+            stream_piece<false, true, true>(A.grad, tbeg, tend, pb, tb, hist, hist + kCells, hist + 2 * kCells, stg,
+                                            kmin, kmax, nf);
+            stg.flush();
+            __syncthreads();
+            flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+            __threadfence();
+            __syncthreads();
+            if (solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
+                             A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, false, smem, S))
+                return;
+            finish_alone(A, t, smem, tb, S);
+        }
+        return;
+    }
+
+    const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
+    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+    for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+        if (tend - tbeg <= kMidN) return;
+        do_round1(t, tbeg, tend, pb_, pe_, false);
     });
     OGQ_CTA_END();
 }
 
-__global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
+__global__ void __launch_bounds__(kSelThreads, 1) k_sel_round2(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ Table tb;
@@ -1181,7 +1257,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
 
     for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
         const int64_t n = tend - tbeg;
-        if (n <= kSmallN) return;
+        if (n <= kMidN) return;
         TState* st = A.ws.st + t;
         if (__ldcg(&st->done)) return;
         __syncthreads();
@@ -1215,12 +1291,12 @@ __global__ void __launch_bounds__(kThreads) k_sel_round2(SelArgs A)
         if (!sh_last) return;
         __threadfence();
         OGQ_CTA_SOLVER(solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme,
-                                    A.s, A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, smem, S));
+                                    A.s, A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, true, smem, S));
     });
     OGQ_CTA_END();
 }
 
-__global__ void __launch_bounds__(kThreads) k_sel_round3(SelArgs A)
+__global__ void __launch_bounds__(kSelThreads, 1) k_sel_round3(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ Table tb;
@@ -1267,7 +1343,7 @@ __global__ void __launch_bounds__(kThreads) k_sel_round3(SelArgs A)
         if (!sh_last) continue;
         __threadfence();
         if (!solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                          A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[1] + tbeg, smem, S))
+                          A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[1] + tbeg, false, smem, S))
             finish_alone(A, t, smem, tb, S);
     }
 }
@@ -1303,8 +1379,8 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
         e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
     }
-    int target = sm_count * 2 < kMaxFlatCtas ? sm_count * 2 : kMaxFlatCtas;
-    FlatGrid g = make_flat_grid(total, target, 16384);
+    int target = sm_count * 4 < kMaxFlatCtas ? sm_count * 4 : kMaxFlatCtas;
+    FlatGrid g = make_flat_grid(total, target, 65536);
     SelArgs A;
     A.grad = d_grad; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
     A.scheme = scheme; A.s = s; A.levels = d_levels; A.status = d_status;
@@ -1312,13 +1388,13 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     cudaError_t e = cudaMemsetAsync(d_ws, 0, sel_zero_bytes(T), stream);
     if (e != cudaSuccess) return e;
     launch_begin("k_sel_round1", stream);
-    k_sel_round1<<<g.ctas + T, kThreads, kSmemBytes, stream>>>(A);
+    k_sel_round1<<<g.ctas + T, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     launch_begin("k_sel_round2", stream);
-    k_sel_round2<<<g.ctas, kThreads, kSmemBytes, stream>>>(A);
+    k_sel_round2<<<g.ctas, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     launch_begin("k_sel_round3", stream);
-    k_sel_round3<<<sm_count * 2, kThreads, kSmemBytes, stream>>>(A);
+    k_sel_round3<<<sm_count, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     return cudaGetLastError();
 }

@@ -340,57 +340,122 @@ OGQ_HD int sel_refine(const SolverView& v, int nr, const int* ra_in, const int* 
     }
     int pa[kMaxIv], pb[kMaxIv];
     int m = 0;
-    int hole = 1;
-    bool use_tight = true;
-    for (;;) {
-        m = 0;
-        bool overflow = false;
-        int idx = 0;
-        while (idx < nr && !overflow) {
-            int hull_b = rb[idx], jn = idx + 1;
-            while (jn < nr && ra[jn] <= hull_b + 1) { if (rb[jn] > hull_b) hull_b = rb[jn]; ++jn; }
-            int iv_j = sel_interval_of_slot(v, ra[idx]);
-            int iv_end = v.slotbase[iv_j] + v.iv[iv_j].ncell;  // end slot of the current interval
-            int run_a = -1, last = -1;
-            bool run_tight = false;
-            for (int c = ra[idx]; c <= hull_b + 1 && !overflow; ++c) {
-                while (c > iv_end && iv_j + 1 < v.m) { ++iv_j; iv_end = v.slotbase[iv_j] + v.iv[iv_j].ncell; }
-                const bool boundary = (c > hull_b) || (c == iv_end);
-                bool populated = false, tight = false;
-                if (!boundary) {
-                    populated = !trim_empty || v.cpre[c + 1] != v.cpre[c];
-                    if (populated && use_tight)
-                        for (int k = idx; k < jn; ++k)
-                            if (ra[k] <= c && c <= rb[k] && rb[k] - ra[k] < kTight) tight = true;
+    // Fast path (the usual case): the ranges do not touch each other, so every range is handled on
+    // its own -- narrow ones by walking their cells, wide sparse ones by hopping from one populated
+    // cell to the next with the prefix counts, wide dense ones by trimming their two ends.
+    bool fast = true;
+    for (int i = 1; i < nr; ++i)
+        if (ra[i] <= rb[i - 1] + 1) fast = false;
+    for (int i = 0; i < nr && fast; ++i) {
+        const int a = ra[i], b = rb[i];
+        int first = a, last = b;
+        bool hop = false;
+        if (trim_empty) {
+            const long long cnt = (long long)v.cpre[b + 1] - (long long)v.cpre[a];
+            if (cnt <= 0) continue;
+            bool gap;
+            first = sel_locate(v, (long long)v.cpre[a], true, &gap);
+            last = sel_locate(v, (long long)v.cpre[b + 1] - 1, false, &gap);
+            if (first < a || last > b || first > last) { fast = false; break; }
+            hop = (last - first + 1 > 12) && cnt <= 32;
+        }
+        if (hop) {
+            // few elements spread over many cells: one piece per populated cell (neighbours joined)
+            long long pos = v.cpre[first];
+            const long long end = v.cpre[last + 1];
+            while (pos < end && fast) {
+                bool gap;
+                const int c = sel_locate(v, pos, true, &gap);
+                if (c < 0 || gap) { fast = false; break; }
+                if (m > 0 && c <= pb[m - 1] + 2 && c > pb[m - 1] &&
+                    sel_interval_of_slot(v, c) == sel_interval_of_slot(v, pb[m - 1])) {
+                    pb[m - 1] = c;
+                } else {
+                    if (m >= kMaxIv) { fast = false; break; }
+                    pa[m] = c; pb[m] = c; ++m;
                 }
-                const bool cut = run_a >= 0 && (boundary || (populated && tight != run_tight) ||
-                                                (!populated && c - last > hole));
-                if (cut) {
-                    if (m >= kMaxIv) overflow = true;
-                    else { pa[m] = run_a; pb[m] = last; ++m; }
+                pos = v.cpre[c + 1];
+            }
+        } else if (last - first + 1 <= 12 && trim_empty) {
+            // narrow: walk the cells, cut at end slots and at more than one empty cell in a row
+            int run_a = -1, lastp = -1;
+            for (int c = first; c <= last + 1 && fast; ++c) {
+                const bool boundary = (c > last) || sel_is_end_slot(v, c);
+                const bool populated = !boundary && v.cpre[c + 1] != v.cpre[c];
+                if (run_a >= 0 && (boundary || (!populated && c - lastp > 1))) {
+                    if (m >= kMaxIv) { fast = false; break; }
+                    pa[m] = run_a; pb[m] = lastp; ++m;
                     run_a = -1;
                 }
-                if (populated) {
-                    if (run_a < 0) { run_a = c; run_tight = tight; }
-                    last = c;
-                }
+                if (populated) { if (run_a < 0) run_a = c; lastp = c; }
             }
-            idx = jn;
+        } else {
+            // wide and dense (or no trimming wanted): the hull, cut where it crosses into another interval
+            int j0 = sel_interval_of_slot(v, first);
+            const int j1 = sel_interval_of_slot(v, last);
+            for (int j = j0; j <= j1 && fast; ++j) {
+                const int lo = v.slotbase[j], hi = v.slotbase[j] + v.iv[j].ncell - 1;
+                const int x = first > lo ? first : lo, y = last < hi ? last : hi;
+                if (x > y) continue;
+                if (m >= kMaxIv) { fast = false; break; }
+                pa[m] = x; pb[m] = y; ++m;
+            }
         }
-        if (!overflow) break;
-        if (hole < (1 << 28)) hole *= 8;
-        else if (use_tight) use_tight = false;
-        else return -11;
+    }
+    if (!fast) {
+        int hole = 1;
+        bool use_tight = true;
+        for (;;) {
+            m = 0;
+            bool overflow = false;
+            int idx = 0;
+            while (idx < nr && !overflow) {
+                int hull_b = rb[idx], jn = idx + 1;
+                while (jn < nr && ra[jn] <= hull_b + 1) { if (rb[jn] > hull_b) hull_b = rb[jn]; ++jn; }
+                int iv_j = sel_interval_of_slot(v, ra[idx]);
+                int iv_end = v.slotbase[iv_j] + v.iv[iv_j].ncell;  // end slot of the current interval
+                int run_a = -1, last = -1;
+                bool run_tight = false;
+                for (int c = ra[idx]; c <= hull_b + 1 && !overflow; ++c) {
+                    while (c > iv_end && iv_j + 1 < v.m) { ++iv_j; iv_end = v.slotbase[iv_j] + v.iv[iv_j].ncell; }
+                    const bool boundary = (c > hull_b) || (c == iv_end);
+                    bool populated = false, tight = false;
+                    if (!boundary) {
+                        populated = !trim_empty || v.cpre[c + 1] != v.cpre[c];
+                        if (populated && use_tight)
+                            for (int k = idx; k < jn; ++k)
+                                if (ra[k] <= c && c <= rb[k] && rb[k] - ra[k] < kTight) tight = true;
+                    }
+                    const bool cut = run_a >= 0 && (boundary || (populated && tight != run_tight) ||
+                                                    (!populated && c - last > hole));
+                    if (cut) {
+                        if (m >= kMaxIv) overflow = true;
+                        else { pa[m] = run_a; pb[m] = last; ++m; }
+                        run_a = -1;
+                    }
+                    if (populated) {
+                        if (run_a < 0) { run_a = c; run_tight = tight; }
+                        last = c;
+                    }
+                }
+                idx = jn;
+            }
+            if (!overflow) break;
+            if (hole < (1 << 28)) hole *= 8;
+            else if (use_tight) use_tight = false;
+            else return -11;
+        }
     }
     if (m == 0) return -12;
     // cell budget: every interval starts with its current cells (always fits), then the spare
     // cells are handed out one halving of the cell width at a time, narrow intervals first
-    int rbits[kMaxIv], order[kMaxIv];
+    int rbits[kMaxIv], order[kMaxIv], psh[kMaxIv];
     {
         int used = 0;
         for (int i = 0; i < m; ++i) {
             rbits[i] = 0;
             order[i] = i;
+            psh[i] = sel_slot_shift(v, pa[i]);
             used += pb[i] - pa[i] + 1;
         }
         if (used > kCells) return -14;
@@ -404,8 +469,7 @@ OGQ_HD int sel_refine(const SolverView& v, int nr, const int* ra_in, const int* 
             changed = false;
             for (int q = 0; q < m; ++q) {
                 const int i = order[q];
-                const int sh = v.iv[sel_interval_of_slot(v, pa[i])].sh;
-                if (rbits[i] >= sh) continue;
+                if (rbits[i] >= psh[i]) continue;
                 const int cost = (pb[i] - pa[i] + 1) << rbits[i];  // extra cells of one more halving
                 if (used + cost > kCells) continue;
                 used += cost;
