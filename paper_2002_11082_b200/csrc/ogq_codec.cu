@@ -17,11 +17,19 @@ namespace ogq {
 constexpr int kMaxLevels = 32;
 constexpr int kMaxWorkers = 64;
 
-// OR-combine the 4*BITS-bit chunk of each lane into words; lane (8q + j), j < BITS,
-// returns word j of 8-lane set q.
+// OR-combine the 4*BITS-bit chunk of each lane into words.  For BITS = 1, 2, 4 a word is made of
+// 8, 4, 2 neighbouring lanes and the first lane of each such set returns it (word index lane / L);
+// for BITS = 3, 5 eight lanes make BITS words and lane (8q + j), j < BITS, returns word j of set q.
 template <int BITS>
 __device__ __forceinline__ uint32_t assemble_words(uint32_t chunk, int lane)
 {
+    if (BITS == 1 || BITS == 2 || BITS == 4) {
+        constexpr int L = 8 / BITS;
+        uint32_t x = chunk << (4 * BITS * (lane & (L - 1)));
+#pragma unroll
+        for (int o = 1; o < L; o <<= 1) x |= __shfl_xor_sync(0xffffffffu, x, o);
+        return x;
+    }
     const int j = lane & 7;
     const int bitpos = j * 4 * BITS;
     const int w0 = bitpos >> 5, sh = bitpos & 31;
@@ -105,15 +113,25 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                     c[j] = (uint32_t)idx + ((lhs < rhs) ? 1u : 0u);
                 }
             }
+            if (i0 + 3 >= n) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j >= n) c[j] = 0u;  // zero padding beyond the tensor
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j >= n) c[j] = 0u;  // zero padding beyond the tensor
+            }
             const uint32_t bits4 = c[0] | (c[1] << BITS) | (c[2] << (2 * BITS)) | (c[3] << (3 * BITS));
             const uint32_t word = assemble_words<BITS>(bits4, lane);
-            const int j8 = lane & 7;
-            if (j8 < BITS) {
-                const int64_t widx = g * (4 * BITS) + (lane >> 3) * BITS + j8;
-                if (widx < region) out[widx] = word;
+            if (BITS == 1 || BITS == 2 || BITS == 4) {
+                constexpr int L = 8 / (BITS == 3 || BITS == 5 ? 1 : BITS);
+                if ((lane & (L - 1)) == 0) {
+                    const int64_t widx = g * (4 * BITS) + lane / L;
+                    if (widx < region) out[widx] = word;
+                }
+            } else {
+                const int j8 = lane & 7;
+                if (j8 < BITS) {
+                    const int64_t widx = g * (4 * BITS) + (lane >> 3) * BITS + j8;
+                    if (widx < region) out[widx] = word;
+                }
             }
         }
     });

@@ -123,7 +123,7 @@ struct Table {  // interval lookup table of the tensor being streamed
     int cellbase[kMaxIv];
     int m, ncells;
     int lo_e;                                      // bottom binade of the round-1 fine window
-    uint32_t prefilter[(kRound1Cells + 31) / 32];  // round-1 cells that touch a candidate interval
+    uint32_t coarse[1024];                         // one bit per block of 2^17 keys that touches an interval
 };
 
 __device__ __forceinline__ void table_from_intervals(Table& tb, const Interval* iv, int m)
@@ -186,18 +186,14 @@ __device__ __forceinline__ void round1_cell(uint32_t bits, int lo_e, bool magnit
 
 __device__ __forceinline__ uint32_t key_to_bits(uint32_t k) { return (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k; }
 
-// Marks every round-1 cell that intersects one of the table's intervals (called by all threads).
-__device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
+// Marks every block of 2^17 keys that intersects one of the table's intervals (called by all threads).
+__device__ __forceinline__ void build_prefilter(Table& tb)
 {
-    for (int i = threadIdx.x; i < (kRound1Cells + 31) / 32; i += kSelThreads) tb.prefilter[i] = 0u;
+    for (int i = threadIdx.x; i < 1024; i += kSelThreads) tb.coarse[i] = 0u;
     __syncthreads();
     if ((int)threadIdx.x < tb.m) {
-        int ca, cb;
-        uint32_t lk;
-        const uint32_t ba = key_to_bits(tb.klo[threadIdx.x]), bb = key_to_bits(tb.khi[threadIdx.x]);
-        round1_cell(magnitude_only ? (ba & 0x7fffffffu) : ba, tb.lo_e, magnitude_only, ca, lk);
-        round1_cell(magnitude_only ? (bb & 0x7fffffffu) : bb, tb.lo_e, magnitude_only, cb, lk);
-        for (int c = ca; c <= cb; ++c) atomicOr(&tb.prefilter[c >> 5], 1u << (c & 31));
+        const uint32_t ba = tb.klo[threadIdx.x] >> 17, bb = tb.khi[threadIdx.x] >> 17;
+        for (uint32_t b = ba; b <= bb; ++b) atomicOr(&tb.coarse[b >> 5], 1u << (b & 31));
     }
     __syncthreads();
 }
@@ -306,6 +302,173 @@ struct Stager {  // per-warp compaction stage
     }
 };
 
+// Block-cooperative visit of grad[pb, pe) without warp collectives: 128-bit loads on the aligned
+// body (four in flight per thread), scalar loads on the ragged head and tail.
+template <class F>
+__device__ __forceinline__ void visit_plain(const float* __restrict__ grad, int64_t pb, int64_t pe, F f)
+{
+    int64_t a = (pb + 3) & ~(int64_t)3;
+    if (a > pe) a = pe;
+    int64_t b = pe & ~(int64_t)3;
+    if (b < a) b = a;
+    const int tid = threadIdx.x;
+    if (tid < (int)(a - pb)) f(__ldg(grad + pb + tid));
+    if (tid < (int)(pe - b)) f(__ldg(grad + b + tid));
+    const float4* g4 = reinterpret_cast<const float4*>(grad);
+    int64_t i = (a >> 2) + tid;
+    const int64_t e = b >> 2;
+    for (; i + 3 * kSelThreads < e; i += 4 * kSelThreads) {
+        const float4 x0 = __ldg(g4 + i);
+        const float4 x1 = __ldg(g4 + i + kSelThreads);
+        const float4 x2 = __ldg(g4 + i + 2 * kSelThreads);
+        const float4 x3 = __ldg(g4 + i + 3 * kSelThreads);
+        f(x0.x); f(x0.y); f(x0.z); f(x0.w);
+        f(x1.x); f(x1.y); f(x1.z); f(x1.w);
+        f(x2.x); f(x2.y); f(x2.z); f(x2.w);
+        f(x3.x); f(x3.y); f(x3.z); f(x3.w);
+    }
+    for (; i < e; i += kSelThreads) {
+        const float4 x = __ldg(g4 + i);
+        f(x.x); f(x.y); f(x.z); f(x.w);
+    }
+}
+
+// Round 1 over grad[pb, pe): per element the round-1 cell (count and low-key-bit sum with carry) and
+// the running min / max key.  Non-finite values show up as extreme keys afterwards.
+__device__ __forceinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe,
+                                              bool magnitude_only, int lo_e, uint32_t* cnt, uint32_t* lo,
+                                              uint32_t* hi, uint32_t& kmin, uint32_t& kmax)
+{
+    const uint32_t lo23 = (uint32_t)lo_e << 23;
+    const uint32_t clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
+    const int base = magnitude_only ? 0 : kRound1Mag;
+    uint32_t mn = kmin, mx = kmax;
+    visit_plain(grad, pb, pe, [&](float v) {
+        uint32_t bits = __float_as_uint(v) & clear;
+        if (bits == 0x80000000u) bits = 0u;
+        const int sgn = (int)bits >> 31;  // 0 or -1
+        const uint32_t mag = bits & 0x7fffffffu;
+        const uint32_t rel = mag - lo23;
+        int mi;
+        uint32_t mask;
+        if (rel < ((uint32_t)kSelW << 23)) {
+            mi = lo_e + (int)(rel >> (23 - kSelM));
+            mask = (1u << (23 - kSelM)) - 1u;
+        } else {
+            const int e = (int)(mag >> 23);
+            mi = (e < lo_e) ? e : e - kSelW + (kSelW << kSelM);
+            mask = 0x7fffffu;
+        }
+        const int cell = base + (mi ^ sgn);
+        const uint32_t lowkey = (mag ^ (uint32_t)sgn) & mask;
+        const uint32_t key = bits ^ ((uint32_t)sgn | 0x80000000u);
+        mn = key < mn ? key : mn;
+        mx = key > mx ? key : mx;
+        atomicAdd(cnt + cell, 1u);
+        const uint32_t old = atomicAdd(lo + cell, lowkey);
+        if (old + lowkey < old) atomicAdd(hi + cell, 1u);
+    });
+    kmin = mn;
+    kmax = mx;
+}
+
+// Round 2 over grad[pb, pe).  Phase A: a one-bit-per-2^17-keys test rejects almost every element;
+// keys that pass are parked in the warp's stage (ballot + popc, no classification yet).  Phase B,
+// whenever the stage fills up: the parked keys are classified exactly 32 at a time, so that the
+// expensive part runs with all lanes busy; keys inside an interval are histogrammed and copied out.
+struct Round2Warp {
+    const Table* tb;
+    uint32_t *cnt, *lo, *hi;
+    uint32_t* stage;
+    uint32_t* dst;
+    unsigned long long* cursor;
+    int fill;
+
+    __device__ __forceinline__ void drain()
+    {
+        const int lane = threadIdx.x & 31;
+        const uint32_t lt = (1u << lane) - 1u;
+        __syncwarp();
+        for (int base = 0; base < fill; base += 32) {
+            const int i = base + lane;
+            uint32_t key = 0;
+            bool in = false;
+            if (i < fill) {
+                key = stage[i];
+                int cell, sh;
+                uint32_t low;
+                in = classify(*tb, key, cell, low, sh);
+                if (in) hist_add(cnt, lo, hi, cell, low);
+            }
+            const uint32_t m2 = __ballot_sync(0xffffffffu, in);
+            if (m2) {
+                unsigned long long pos = 0;
+                if (lane == 0) pos = atomicAdd(cursor, (unsigned long long)__popc(m2));
+                pos = __shfl_sync(0xffffffffu, pos, 0);
+                if (in) dst[pos + __popc(m2 & lt)] = key;
+            }
+        }
+        __syncwarp();
+        fill = 0;
+    }
+
+    __device__ __forceinline__ void park(uint32_t key, bool maybe)
+    {
+        const uint32_t m = __ballot_sync(0xffffffffu, maybe);
+        if (m) {
+            const int lane = threadIdx.x & 31;
+            if (maybe) stage[fill + __popc(m & ((1u << lane) - 1u))] = key;
+            fill += __popc(m);
+            if (fill > kStageCap - 32) drain();
+        }
+    }
+};
+
+__device__ __forceinline__ void stream_round2(const float* __restrict__ grad, int64_t pb, int64_t pe,
+                                              bool magnitude_only, const Table& tb, uint32_t* cnt, uint32_t* lo,
+                                              uint32_t* hi, uint32_t* stage, uint32_t* dst,
+                                              unsigned long long* cursor)
+{
+    const uint32_t clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    Round2Warp w;
+    w.tb = &tb; w.cnt = cnt; w.lo = lo; w.hi = hi; w.stage = stage; w.dst = dst; w.cursor = cursor; w.fill = 0;
+    auto one = [&](float v, bool valid) {
+        uint32_t bits = __float_as_uint(v) & clear;
+        if (bits == 0x80000000u) bits = 0u;
+        const uint32_t key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
+        const uint32_t blk = key >> 17;
+        w.park(key, valid && ((tb.coarse[blk >> 5] >> (blk & 31)) & 1u));
+    };
+    int64_t a = (pb + 3) & ~(int64_t)3;
+    if (a > pe) a = pe;
+    int64_t b = pe & ~(int64_t)3;
+    if (b < a) b = a;
+    if (warp == 0) {  // ragged head and tail, one element per lane
+        float v = 0.f;
+        bool valid = false;
+        if (lane < (int)(a - pb)) { v = __ldg(grad + pb + lane); valid = true; }
+        else if (lane >= 4 && lane - 4 < (int)(pe - b)) { v = __ldg(grad + b + lane - 4); valid = true; }
+        one(v, valid);
+    }
+    const float4* g4 = reinterpret_cast<const float4*>(grad);
+    const int64_t e = b >> 2;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t i0 = (a >> 2) + warp * 32; i0 < e; i0 += 4 * kSelThreads) {  // trip count is warp-uniform
+        const int64_t i = i0 + lane;
+        const bool ok0 = i < e, ok1 = i + kSelThreads < e, ok2 = i + 2 * kSelThreads < e, ok3 = i + 3 * kSelThreads < e;
+        const float4 x0 = ok0 ? __ldg(g4 + i) : zero;
+        const float4 x1 = ok1 ? __ldg(g4 + i + kSelThreads) : zero;
+        const float4 x2 = ok2 ? __ldg(g4 + i + 2 * kSelThreads) : zero;
+        const float4 x3 = ok3 ? __ldg(g4 + i + 3 * kSelThreads) : zero;
+        one(x0.x, ok0); one(x0.y, ok0); one(x0.z, ok0); one(x0.w, ok0);
+        one(x1.x, ok1); one(x1.y, ok1); one(x1.z, ok1); one(x1.w, ok1);
+        one(x2.x, ok2); one(x2.y, ok2); one(x2.z, ok2); one(x2.w, ok2);
+        one(x3.x, ok3); one(x3.y, ok3); one(x3.z, ok3); one(x3.w, ok3);
+    }
+    w.drain();
+}
+
 // Streams one piece of a tensor's working set: histogram of the keys inside the intervals,
 // optional copy of those keys, and (round 1) min / max / non-finite tracking.
 template <bool FIRST, bool FROM_GRAD, bool COMPACT>
@@ -322,34 +485,8 @@ __device__ __forceinline__ void stream_piece(const void* __restrict__ src, int64
             if (COMPACT) kk[c++] = key;
         }
     };
-    if (FROM_GRAD) {
-        warp_visit4<float4, float>((const float*)src, pb, pe, [&](const float* x, int nv) {
-            uint32_t kk[4];
-            int c = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (j < nv) {
-                    uint32_t bits = __float_as_uint(x[j]);
-                    if (magnitude_only) bits &= 0x7fffffffu;
-                    else if (bits == 0x80000000u) bits = 0u;
-                    int cell;
-                    uint32_t low;
-                    round1_cell(bits, tb.lo_e, magnitude_only, cell, low);
-                    if (FIRST) {
-                        if ((bits & 0x7f800000u) == 0x7f800000u) nonfinite = 1u;
-                        const uint32_t key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
-                        kmin = key < kmin ? key : kmin;
-                        kmax = key > kmax ? key : kmax;
-                        hist_add(cnt, lo, hi, cell, low);
-                    } else if ((tb.prefilter[cell >> 5] >> (cell & 31)) & 1u) {
-                        const uint32_t key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
-                        handle(key, kk, c);
-                    }
-                }
-            }
-            if (COMPACT) stg.append(kk, c);
-        });
-    } else {
+    static_assert(!FROM_GRAD && !FIRST, "fp32 input goes through stream_round1 / stream_round2");
+    {
         warp_visit4<uint4, uint32_t>((const uint32_t*)src, pb, pe, [&](const uint32_t* x, int nv) {
             uint32_t kk[4];
             int c = 0;
@@ -1118,11 +1255,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
         __syncthreads();
         zero_hist(hist, tb.ncells);
         __syncthreads();
-        Stager stg;
-        stg.stage = nullptr; stg.dst = nullptr; stg.cursor = nullptr; stg.fill = 0;
         uint32_t kmin = 0xffffffffu, kmax = 0u, nf = 0u;
-        stream_piece<true, true, false>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stg,
-                                        kmin, kmax, nf);
+        stream_round1(A.grad, pb_, pe_, pb, tb.lo_e, hist, hist + kCells, hist + 2 * kCells, kmin, kmax);
+        nf = (kmax >= 0xff800000u || kmin <= 0x007fffffu) ? 1u : 0u;  // Inf / NaN keys lie beyond these
         // combine min / max / non-finite over the CTA, then one atomic each
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -1210,18 +1345,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
                 tb.lo_e = st->hi_e - kSelW;
             }
             __syncthreads();
-            build_prefilter(tb, pb);
+            build_prefilter(tb);
             zero_hist(hist, tb.ncells);
             __syncthreads();
-            Stager stg;
-            stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
-            stg.dst = A.ws.buf[0] + tbeg;
-            stg.cursor = &st->cursor[0];
-            stg.fill = 0;
-            uint32_t kmin = 0, kmax = 0, nf = 0;
-            stream_piece<false, true, true>(A.grad, tbeg, tend, pb, tb, hist, hist + kCells, hist + 2 * kCells, stg,
-                                            kmin, kmax, nf);
-            stg.flush();
+            stream_round2(A.grad, tbeg, tend, pb, tb, hist, hist + kCells, hist + 2 * kCells,
+                          reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
+                          A.ws.buf[0] + tbeg, &st->cursor[0]);
             __syncthreads();
             flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
             __threadfence();
@@ -1266,18 +1395,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round2(SelArgs A)
             tb.lo_e = st->hi_e - kSelW;
         }
         __syncthreads();
-        build_prefilter(tb, pb);
+        build_prefilter(tb);
         zero_hist(hist, tb.ncells);
         __syncthreads();
-        Stager stg;
-        stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
-        stg.dst = A.ws.buf[0] + tbeg;
-        stg.cursor = &st->cursor[0];
-        stg.fill = 0;
-        uint32_t kmin = 0, kmax = 0, nf = 0;
-        stream_piece<false, true, true>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stg,
-                                        kmin, kmax, nf);
-        stg.flush();
+        stream_round2(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells,
+                      reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
+                      A.ws.buf[0] + tbeg, &st->cursor[0]);
         __syncthreads();
         flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         __threadfence();
