@@ -104,8 +104,10 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                 const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
+                    // s = 2^(BITS-1) + 1 levels (s = 2 for BITS = 1): BITS - 1 halving steps
                     int idx = 0;
-                    for (int step = (s - 1) >> 1; step >= 1; step >>= 1)
+#pragma unroll
+                    for (int step = (BITS >= 2) ? (1 << (BITS - 2)) : 0; step >= 1; step >>= 1)
                         if (sh_lv[idx + step] <= x[j]) idx += step;
                     const float d = __fsub_rn(x[j], sh_lv[idx]);
                     const float lhs = __fmul_rn((float)(rw[j] >> 8), sh_w[idx + 1]);

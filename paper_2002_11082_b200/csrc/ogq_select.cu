@@ -335,26 +335,22 @@ __device__ __forceinline__ void visit_plain(const float* __restrict__ grad, int6
 
 // Round 1 over grad[pb, pe): per element the round-1 cell (count and low-key-bit sum with carry) and
 // the running min / max key.  Non-finite values show up as extreme keys afterwards.
-__device__ __forceinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe,
-                                              bool magnitude_only, int lo_e, uint32_t* cnt, uint32_t* lo,
-                                              uint32_t* hi, uint32_t& kmin, uint32_t& kmax)
-{
-    const uint32_t lo23 = (uint32_t)lo_e << 23;
-    const uint32_t clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
-    const int base = magnitude_only ? 0 : kRound1Mag;
-    uint32_t mn = kmin, mx = kmax;
-    visit_plain(grad, pb, pe, [&](float v) {
+struct Round1Body {
+    uint32_t lo23, clear;
+    int lo_e, base;
+    uint32_t *cnt, *lo, *hi;
+    uint32_t mn, mx;
+
+    __device__ __forceinline__ void operator()(float v)
+    {
         uint32_t bits = __float_as_uint(v) & clear;
         if (bits == 0x80000000u) bits = 0u;
         const int sgn = (int)bits >> 31;  // 0 or -1
         const uint32_t mag = bits & 0x7fffffffu;
         const uint32_t rel = mag - lo23;
-        int mi;
-        uint32_t mask;
-        if (rel < ((uint32_t)kSelW << 23)) {
-            mi = lo_e + (int)(rel >> (23 - kSelM));
-            mask = (1u << (23 - kSelM)) - 1u;
-        } else {
+        int mi = lo_e + (int)(rel >> (23 - kSelM));
+        uint32_t mask = (1u << (23 - kSelM)) - 1u;
+        if (rel >= ((uint32_t)kSelW << 23)) {  // outside the fine window: one cell per binade
             const int e = (int)(mag >> 23);
             mi = (e < lo_e) ? e : e - kSelW + (kSelW << kSelM);
             mask = 0x7fffffu;
@@ -367,9 +363,43 @@ __device__ __forceinline__ void stream_round1(const float* __restrict__ grad, in
         atomicAdd(cnt + cell, 1u);
         const uint32_t old = atomicAdd(lo + cell, lowkey);
         if (old + lowkey < old) atomicAdd(hi + cell, 1u);
-    });
-    kmin = mn;
-    kmax = mx;
+    }
+};
+
+__device__ __forceinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe,
+                                              bool magnitude_only, int lo_e, uint32_t* cnt, uint32_t* lo,
+                                              uint32_t* hi, uint32_t& kmin, uint32_t& kmax)
+{
+    Round1Body f;
+    f.lo23 = (uint32_t)lo_e << 23;
+    f.clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
+    f.lo_e = lo_e;
+    f.base = magnitude_only ? 0 : kRound1Mag;
+    f.cnt = cnt; f.lo = lo; f.hi = hi;
+    f.mn = kmin; f.mx = kmax;
+    int64_t a = (pb + 3) & ~(int64_t)3;
+    if (a > pe) a = pe;
+    int64_t b = pe & ~(int64_t)3;
+    if (b < a) b = a;
+    const int tid = threadIdx.x;
+    if (tid < (int)(a - pb)) f(__ldg(grad + pb + tid));
+    if (tid < (int)(pe - b)) f(__ldg(grad + b + tid));
+    const float4* g4 = reinterpret_cast<const float4*>(grad);
+    int64_t i = (a >> 2) + tid;
+    const int64_t e = b >> 2;
+    for (; i + 3 * kSelThreads < e; i += 4 * kSelThreads) {
+        float4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i + u * kSelThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { f(x[u].x); f(x[u].y); f(x[u].z); f(x[u].w); }
+    }
+    for (; i < e; i += kSelThreads) {
+        const float4 x = __ldg(g4 + i);
+        f(x.x); f(x.y); f(x.z); f(x.w);
+    }
+    kmin = f.mn;
+    kmax = f.mx;
 }
 
 // Round 2 over grad[pb, pe).  Phase A: a one-bit-per-2^17-keys test rejects almost every element;
@@ -384,7 +414,7 @@ struct Round2Warp {
     unsigned long long* cursor;
     int fill;
 
-    __device__ __forceinline__ void drain()
+    __device__ __noinline__ void drain()
     {
         const int lane = threadIdx.x & 31;
         const uint32_t lt = (1u << lane) - 1u;
@@ -412,6 +442,17 @@ struct Round2Warp {
         fill = 0;
     }
 
+    uint32_t clear;
+
+    __device__ __forceinline__ void one(float v, bool valid)
+    {
+        uint32_t bits = __float_as_uint(v) & clear;
+        if (bits == 0x80000000u) bits = 0u;
+        const uint32_t key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
+        const uint32_t blk = key >> 17;
+        park(key, valid && ((tb->coarse[blk >> 5] >> (blk & 31)) & 1u));
+    }
+
     __device__ __forceinline__ void park(uint32_t key, bool maybe)
     {
         const uint32_t m = __ballot_sync(0xffffffffu, maybe);
@@ -433,13 +474,7 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     Round2Warp w;
     w.tb = &tb; w.cnt = cnt; w.lo = lo; w.hi = hi; w.stage = stage; w.dst = dst; w.cursor = cursor; w.fill = 0;
-    auto one = [&](float v, bool valid) {
-        uint32_t bits = __float_as_uint(v) & clear;
-        if (bits == 0x80000000u) bits = 0u;
-        const uint32_t key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
-        const uint32_t blk = key >> 17;
-        w.park(key, valid && ((tb.coarse[blk >> 5] >> (blk & 31)) & 1u));
-    };
+    w.clear = clear;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
     int64_t b = pe & ~(int64_t)3;
@@ -449,22 +484,23 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
         bool valid = false;
         if (lane < (int)(a - pb)) { v = __ldg(grad + pb + lane); valid = true; }
         else if (lane >= 4 && lane - 4 < (int)(pe - b)) { v = __ldg(grad + b + lane - 4); valid = true; }
-        one(v, valid);
+        w.one(v, valid);
     }
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     const int64_t e = b >> 2;
-    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int64_t i0 = (a >> 2) + warp * 32; i0 < e; i0 += 4 * kSelThreads) {  // trip count is warp-uniform
-        const int64_t i = i0 + lane;
-        const bool ok0 = i < e, ok1 = i + kSelThreads < e, ok2 = i + 2 * kSelThreads < e, ok3 = i + 3 * kSelThreads < e;
-        const float4 x0 = ok0 ? __ldg(g4 + i) : zero;
-        const float4 x1 = ok1 ? __ldg(g4 + i + kSelThreads) : zero;
-        const float4 x2 = ok2 ? __ldg(g4 + i + 2 * kSelThreads) : zero;
-        const float4 x3 = ok3 ? __ldg(g4 + i + 3 * kSelThreads) : zero;
-        one(x0.x, ok0); one(x0.y, ok0); one(x0.z, ok0); one(x0.w, ok0);
-        one(x1.x, ok1); one(x1.y, ok1); one(x1.z, ok1); one(x1.w, ok1);
-        one(x2.x, ok2); one(x2.y, ok2); one(x2.z, ok2); one(x2.w, ok2);
-        one(x3.x, ok3); one(x3.y, ok3); one(x3.z, ok3); one(x3.w, ok3);
+        float4 x[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t i = i0 + lane + (int64_t)u * kSelThreads;
+            ok[u] = i < e;
+            x[u] = ok[u] ? __ldg(g4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            w.one(x[u].x, ok[u]); w.one(x[u].y, ok[u]); w.one(x[u].z, ok[u]); w.one(x[u].w, ok[u]);
+        }
     }
     w.drain();
 }
@@ -580,6 +616,8 @@ struct SolverShared {
     int done, nm, internal;
     uint32_t offc[kMaxIv];    // per-interval shifts of the scanned prefix arrays
     double offs[kMaxIv];
+    int nr, ra[kMaxLv], rb[kMaxLv];  // open slot ranges of this pass
+    int pa[kMaxIv], pb[kMaxIv];      // pieces cut out of them
     long long cand;           // elements inside the new intervals
     int n_keys, n_unique;     // sorting finish
     int ivstart[kMaxIv], ivufirst[kMaxIv];
@@ -718,7 +756,6 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        int stbits = 0;
         int next = S.n_unique;
         for (int j = S.nm - 1; j >= 0; --j) {
             if (S.ivufirst[j] < 0) {  // no element left in this interval: only its end slot
@@ -731,23 +768,148 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
         }
         int cb = 0;
         for (int j = 0; j < S.nm; ++j) { S.niv[j].sh = 0; S.niv[j].cellbase = cb; cb += S.niv[j].ncell; }
-        SolverView xv;
-        xv.slot_iv = nullptr; xv.xkeys = xkeys; xv.cpre = xcpre; xv.spre = xspre; xv.iv = S.niv; xv.m = S.nm;
-        xv.n = S.view.n; xv.stot = S.view.stot;
-        sel_init_slots(xv);
-        int ra[kMaxLv], rb[kMaxLv];
-        int open = (S.n_keys > kSmallN) ? -1 : sel_orq_pass(xv, s, S.lv, ra, rb);
-        if (open == 0) {
+        S.view.slot_iv = nullptr; S.view.xkeys = xkeys; S.view.cpre = xcpre; S.view.spre = xspre;
+        S.view.iv = S.niv; S.view.m = S.nm;
+        sel_init_slots(S.view);
+        S.internal = (S.n_keys > kSmallN) ? 1 : 0;
+    }
+    // one thread per level, one depth at a time (every cell is a single key now, so each solve is exact)
+    for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
+        __syncthreads();
+        const int q = threadIdx.x;
+        if (!S.internal && q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0 && !S.lv[q].exact) {
+            if (!sel_orq_solve(S.view, S.lv[q - stride], S.lv[q + stride], S.lv[q])) S.internal = 1;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool ok = !S.internal;
+        for (int q = 0; q < s; ++q) ok = ok && S.lv[q].exact;
+        if (ok) {
             for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = sel_key_to_float(S.lv[q].key);
         } else {
-            stbits = OGQ_ST_INTERNAL;
+            status[t] |= OGQ_ST_INTERNAL;
             for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
         }
-        if (stbits) status[t] |= stbits;
         st->done = 1;
         __threadfence();
     }
     __syncthreads();
+}
+
+// Warp-parallel version of the common case of sel_refine: the open ranges are sorted and do not
+// touch, every range yields at most four pieces, there are at most 32 pieces and none is wider
+// than an equal share of the cell budget.  Lane i first cuts range i into pieces, then lane k
+// builds interval k.  Returns false (nothing written) when the case is not the common one; the
+// caller then runs the general single-thread routine.  Called by the 32 lanes of warp 0.
+__device__ bool refine_parallel(SolverShared& S, bool trim_empty)
+{
+    const SolverView& v = S.view;
+    const int lane = threadIdx.x & 31;
+    const int nr = S.nr;
+    int p_a[4], p_b[4], np = 0;
+    bool fail = nr > 32;
+    if (lane < nr && !fail) {
+        const int a = S.ra[lane], b = S.rb[lane];
+        if (lane > 0 && a <= S.rb[lane - 1] + 1) fail = true;
+        int first = a, last = b;
+        long long cnt = 1;
+        if (trim_empty) {
+            cnt = (long long)v.cpre[b + 1] - (long long)v.cpre[a];
+            if (cnt > 0) {
+                bool gap;
+                first = sel_locate(v, (long long)v.cpre[a], true, &gap);
+                last = sel_locate(v, (long long)v.cpre[b + 1] - 1, false, &gap);
+                if (first < a || last > b || first > last) fail = true;
+            }
+        }
+        if (cnt > 0 && !fail) {
+            const int width = last - first + 1;
+            if (trim_empty && width <= 12) {
+                int run_a = -1, lastp = -1;
+                for (int c = first; c <= last + 1; ++c) {
+                    const bool boundary = (c > last) || sel_is_end_slot(v, c);
+                    const bool populated = !boundary && v.cpre[c + 1] != v.cpre[c];
+                    if (run_a >= 0 && (boundary || (!populated && c - lastp > 1))) {
+                        if (np >= 4) { fail = true; break; }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) if (u == np) { p_a[u] = run_a; p_b[u] = lastp; }
+                        ++np;
+                        run_a = -1;
+                    }
+                    if (populated) { if (run_a < 0) run_a = c; lastp = c; }
+                }
+            } else {
+                // wide: the trimmed hull, cut where it crosses into another interval (if it is too wide
+                // for its share of the cells the general routine takes over below)
+                const int j0 = sel_interval_of_slot(v, first), j1 = sel_interval_of_slot(v, last);
+                for (int j = j0; j <= j1; ++j) {
+                    const int lo = v.slotbase[j], hi = v.slotbase[j] + v.iv[j].ncell - 1;
+                    const int x = first > lo ? first : lo, y = last < hi ? last : hi;
+                    if (x > y) continue;
+                    if (np >= 4) { fail = true; break; }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) if (u == np) { p_a[u] = x; p_b[u] = y; }
+                    ++np;
+                }
+            }
+        }
+    }
+    if (__any_sync(0xffffffffu, fail)) return false;
+    // piece offsets
+    int incl = np;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += nb;
+    }
+    const int m = __shfl_sync(0xffffffffu, incl, 31);
+    if (m == 0 || m > 32) return false;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        if (u < np) { S.pa[incl - np + u] = p_a[u]; S.pb[incl - np + u] = p_b[u]; }
+    __syncwarp();
+    // one lane per piece: equal share of the cell budget
+    const int share = kCells / m;
+    int cells = 0, sh = 0, r = 0, j = 0, pa = 0, pb = 0;
+    long long elems = 0;
+    if (lane < m) {
+        pa = S.pa[lane]; pb = S.pb[lane];
+        cells = pb - pa + 1;
+        j = sel_interval_of_slot(v, pa);
+        sh = v.iv[j].sh;
+        r = (cells <= share) ? sel_floor_log2(share / cells) : -1;
+        if (r > sh) r = sh;
+        elems = (long long)v.cpre[pb + 1] - (long long)v.cpre[pa];
+    }
+    if (__any_sync(0xffffffffu, lane < m && r < 0)) return false;  // a piece wider than its share
+    const int ncell = (lane < m) ? (cells << r) : 0;
+    int cinc = ncell;
+    long long einc = elems;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int nb = __shfl_up_sync(0xffffffffu, cinc, o);
+        const long long eb = __shfl_up_sync(0xffffffffu, einc, o);
+        if (lane >= o) { cinc += nb; einc += eb; }
+    }
+    const bool progress = __any_sync(0xffffffffu, lane < m && r > 0);
+    const bool open_shift = __any_sync(0xffffffffu, lane < m && sh - r > 0);
+    if (open_shift && !progress) return false;
+    if (lane < m) {
+        const Interval& o = v.iv[j];
+        Interval& ni = S.niv[lane];
+        ni.sh = sh - r;
+        ni.ncell = ncell;
+        ni.klo = o.klo + ((uint32_t)(pa - v.slotbase[j]) << o.sh);
+        ni.khi = ni.klo + (uint32_t)((((unsigned long long)ncell) << ni.sh) - 1ull);
+        ni.cellbase = cinc - ncell;
+        ni.pad = 0;
+        ni.cbefore = v.cpre[pa];
+        ni.sbefore = v.spre[pa];
+    }
+    if (lane == 31) { S.cand = einc; S.nm = m; }
+    __syncwarp();
+    return true;
 }
 
 // Runs one solver pass for tensor t after all of its pieces of the current round arrived.
@@ -905,7 +1067,6 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     OGQ_TICK(st, 2);
 
     if (threadIdx.x == 0) {
-        int ra[kMaxLv], rb[kMaxLv];
         int open = 0;
         int stbits = 0;
         if (S.internal) {
@@ -929,41 +1090,53 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
                     levels[2 * t] = -b1; levels[2 * t + 1] = b1;
                     S.done = 1;
                 } else {
-                    ra[0] = a; rb[0] = b; open = 1;
+                    S.ra[0] = a; S.rb[0] = b; open = 1;
                 }
             }
         } else {
             for (int q = 1; q < s - 1; ++q)
-                if (!S.lv[q].exact) { ra[open] = S.lv[q].sa; rb[open] = S.lv[q].sb; ++open; }
-            if (open == 0) {
-                for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = sel_key_to_float(S.lv[q].key);
-                S.done = 1;
-            } else {
-                for (int q = 0; q < s; ++q) {
-                    ExactLv& e = st->lv[q];
-                    e.exact = S.lv[q].exact; e.key = S.lv[q].key;
-                    e.c_lt = S.lv[q].c_lt; e.c_le = S.lv[q].c_le; e.s_lt = S.lv[q].s_lt; e.s_le = S.lv[q].s_le;
-                }
-            }
+                if (!S.lv[q].exact) { S.ra[open] = S.lv[q].sa; S.rb[open] = S.lv[q].sb; ++open; }
+            if (open == 0) S.done = 1;
         }
-        if (!S.done) {
-            S.cand = 0;
-            const int nm = (round + 1 > kMaxRounds) ? -2 : sel_refine(S.view, open, ra, rb, !pb, S.niv, &S.cand);
+        S.nr = open;
+        S.nm = -100;
+        S.cand = 0;
+        if (!S.done && round + 1 > kMaxRounds) { stbits = OGQ_ST_ITER_CAP; S.done = 1; }
+        if (stbits) {
+            // unresolved: leave zeros rather than garbage
+            if (pb) { levels[2 * t] = 0.f; levels[2 * t + 1] = 0.f; }
+            else for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
+            status[t] |= stbits;
+        }
+    }
+    __syncthreads();
+    if (!pb && !S.internal && (int)threadIdx.x < s) {
+        if (S.done) {
+            if (S.nr == 0 && !(status[t] & (OGQ_ST_ITER_CAP | OGQ_ST_INTERNAL)))
+                levels[(int64_t)t * s + threadIdx.x] = sel_key_to_float(S.lv[threadIdx.x].key);
+        } else {
+            ExactLv& e = st->lv[threadIdx.x];
+            const LvInfo& l = S.lv[threadIdx.x];
+            e.exact = l.exact; e.key = l.key; e.c_lt = l.c_lt; e.c_le = l.c_le; e.s_lt = l.s_lt; e.s_le = l.s_le;
+        }
+    }
+    if (!S.done) {
+        // intervals of the next round: warp-parallel common case, single-thread general case
+        bool ok = true;
+        if (threadIdx.x < 32) ok = refine_parallel(S, !pb);
+        if (threadIdx.x == 0 && !ok) {
+            const int nm = sel_refine(S.view, S.nr, S.ra, S.rb, !pb, S.niv, &S.cand);
             if (nm < 0) {
-                stbits = (nm == -2) ? OGQ_ST_ITER_CAP : OGQ_ST_INTERNAL;
+                if (pb) { levels[2 * t] = 0.f; levels[2 * t + 1] = 0.f; }
+                else for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
+                status[t] |= OGQ_ST_INTERNAL;
                 S.done = 1;
             } else {
                 S.nm = nm;
             }
         }
-        if (S.done && stbits) {
-            // unresolved: leave zeros rather than garbage
-            if (pb) { levels[2 * t] = 0.f; levels[2 * t + 1] = 0.f; }
-            else for (int q = 0; q < s; ++q) levels[(int64_t)t * s + q] = 0.f;
-        }
-        if (stbits) status[t] |= stbits;
-        OGQ_TICK(st, 3);
     }
+    OGQ_TICK(st, 3);
     __syncthreads();
 
     if (S.done) {
