@@ -217,25 +217,54 @@ def run_ours(args):
     status = [torch.zeros((T,), dtype=torch.int32, device=dev) for _ in range(K)]
     packed = [torch.zeros((int(h_po[-1]),), dtype=torch.int32, device=dev) for _ in range(K)]
     ws_bytes = ogq.ogq_workspace_bytes(T, N, max(s, 3))
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    # workers alternate between `args.streams` CUDA streams, each with its own scratch, so that the
+    # short single-CTA solver tails of one worker overlap the streaming kernels of the next
+    n_streams = max(1, min(args.streams, K))
+    wss = [torch.empty(ws_bytes, dtype=torch.uint8, device=dev) for _ in range(n_streams)]
+    side = [torch.cuda.Stream(device=dev) for _ in range(n_streams)] if n_streams > 1 else []
     out = torch.empty(N, device=dev)
     pk_ptrs = ogq.device_pointer_array(packed)
     lv_ptrs = ogq.device_pointer_array(levels)
 
-    def lqp(k):
+    def lqp(k, stream=None):
+        ws = wss[k % n_streams]
         if scheme == ogq.OGQ_ORQ:
-            ogq.ogq_levels_orq(grads[k], off, T, N, s, levels[k], status[k], ws, ws_bytes)
-            ogq.ogq_quantize_pack(grads[k], off, T, N, scheme, s, levels[k], None, args.seed, k, po, packed[k])
+            ogq.ogq_levels_orq(grads[k], off, T, N, s, levels[k], status[k], ws, ws_bytes, stream)
+            ogq.ogq_quantize_pack(grads[k], off, T, N, scheme, s, levels[k], None, args.seed, k, po, packed[k], stream)
         else:
-            ogq.ogq_levels_bingrad(grads[k], off, T, N, scheme, lloyd, levels[k], thresh[k], status[k], ws, ws_bytes)
-            ogq.ogq_quantize_pack(grads[k], off, T, N, scheme, 2, levels[k], thresh[k], args.seed, k, po, packed[k])
+            ogq.ogq_levels_bingrad(grads[k], off, T, N, scheme, lloyd, levels[k], thresh[k], status[k], ws, ws_bytes,
+                                   stream)
+            ogq.ogq_quantize_pack(grads[k], off, T, N, scheme, 2, levels[k], thresh[k], args.seed, k, po, packed[k],
+                                  stream)
 
     def unpack():
         ogq.ogq_unpack_sum(pk_ptrs, lv_ptrs, K, off, po, T, N, s, 1.0 / K, out)
 
-    def step():
+    def lqp_all(before=None):
+        """levels + quantize + pack of all K workers; `before(k)` runs on worker k's stream first."""
+        if n_streams == 1:
+            for k in range(K):
+                if before is not None:
+                    before(k)
+                lqp(k)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        for st in side:
+            st.wait_event(fork)
         for k in range(K):
-            lqp(k)
+            with torch.cuda.stream(side[k % n_streams]):
+                if before is not None:
+                    before(k)
+                lqp(k, side[k % n_streams])
+        for st in side:
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
+
+    def step():
+        lqp_all()
         unpack()
 
     def barrier():
@@ -280,12 +309,14 @@ def run_ours(args):
     value = world * grad_bytes / (ms_step * 1e-3) / 1e9
 
     # ---- per-stage and per-kernel times (separate instrumented passes, not part of `value`)
-    ms_lqp = timed(lambda: [lqp(k) for k in range(K)], steps) / steps
+    ms_lqp = timed(lqp_all, steps) / steps
     ms_unp = timed(unpack, steps) / steps
-    ogq.ogq_profile_enable(True)
+    ogq.ogq_profile_enable(True)  # per-kernel times: one stream, so that no two kernels overlap
     torch.cuda.synchronize()
     for _ in range(steps):
-        step()
+        for k in range(K):
+            lqp(k)
+        unpack()
     torch.cuda.synchronize()
     recs = ogq.ogq_profile_collect()
     ogq.ogq_profile_enable(False)
@@ -319,9 +350,7 @@ def run_ours(args):
         h_out = torch.empty(N, dtype=torch.float32).pin_memory()
 
         def e2e_step():
-            for k in range(K):
-                grads[k].copy_(pinned[k], non_blocking=True)
-                lqp(k)
+            lqp_all(before=lambda k: grads[k].copy_(pinned[k], non_blocking=True))
             unpack()
             h_out.copy_(out, non_blocking=True)
 
@@ -347,7 +376,7 @@ def run_ours(args):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "scheme": args.scheme, "levels": s, "bits": bits,
-                       "workers_per_gpu": K, "tensors": T, "elements": N,
+                       "workers_per_gpu": K, "tensors": T, "elements": N, "streams": n_streams,
                        "l2": "inputs larger than L2 (no flush)" if 4 * N * K > 2 * 126e6 else "working set near L2 size; no flush"},
             "stages": {
                 "levels_quantize_pack": {"ms": ms_lqp, "grad_gbs": grad_bytes / (ms_lqp * 1e-3) / 1e9,
@@ -373,6 +402,7 @@ def main():
     ap.add_argument("--scheme", default="orq9", choices=sorted(SCHEMES))
     ap.add_argument("--workers", type=int, default=8)
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--streams", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
