@@ -338,7 +338,7 @@ __device__ __forceinline__ void visit_plain(const float* __restrict__ grad, int6
 struct Round1Body {
     uint32_t lo23, clear;
     int lo_e, base;
-    uint32_t *cnt, *lo, *hi;
+    uint32_t* hist;  // counts at [0, kCells), low sums at [kCells, 2 kCells), carries above
     uint32_t mn, mx;
 
     __device__ __forceinline__ void operator()(float v)
@@ -360,9 +360,9 @@ struct Round1Body {
         const uint32_t key = bits ^ ((uint32_t)sgn | 0x80000000u);
         mn = key < mn ? key : mn;
         mx = key > mx ? key : mx;
-        atomicAdd(cnt + cell, 1u);
-        const uint32_t old = atomicAdd(lo + cell, lowkey);
-        if (old + lowkey < old) atomicAdd(hi + cell, 1u);
+        atomicAdd(hist + cell, 1u);
+        const uint32_t old = atomicAdd(hist + kCells + cell, lowkey);
+        if (old + lowkey < old) atomicAdd(hist + 2 * kCells + cell, 1u);
     }
 };
 
@@ -375,7 +375,7 @@ __device__ __forceinline__ void stream_round1(const float* __restrict__ grad, in
     f.clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
     f.lo_e = lo_e;
     f.base = magnitude_only ? 0 : kRound1Mag;
-    f.cnt = cnt; f.lo = lo; f.hi = hi;
+    f.hist = cnt;
     f.mn = kmin; f.mx = kmax;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
@@ -406,42 +406,46 @@ __device__ __forceinline__ void stream_round1(const float* __restrict__ grad, in
 // keys that pass are parked in the warp's stage (ballot + popc, no classification yet).  Phase B,
 // whenever the stage fills up: the parked keys are classified exactly 32 at a time, so that the
 // expensive part runs with all lanes busy; keys inside an interval are histogrammed and copied out.
-struct Round2Warp {
-    const Table* tb;
+struct Round2Ctx {  // per-CTA constants of round 2, kept in shared memory to spare registers
     uint32_t *cnt, *lo, *hi;
-    uint32_t* stage;
     uint32_t* dst;
     unsigned long long* cursor;
-    int fill;
+};
 
-    __device__ __noinline__ void drain()
-    {
-        const int lane = threadIdx.x & 31;
-        const uint32_t lt = (1u << lane) - 1u;
-        __syncwarp();
-        for (int base = 0; base < fill; base += 32) {
-            const int i = base + lane;
-            uint32_t key = 0;
-            bool in = false;
-            if (i < fill) {
-                key = stage[i];
-                int cell, sh;
-                uint32_t low;
-                in = classify(*tb, key, cell, low, sh);
-                if (in) hist_add(cnt, lo, hi, cell, low);
-            }
-            const uint32_t m2 = __ballot_sync(0xffffffffu, in);
-            if (m2) {
-                unsigned long long pos = 0;
-                if (lane == 0) pos = atomicAdd(cursor, (unsigned long long)__popc(m2));
-                pos = __shfl_sync(0xffffffffu, pos, 0);
-                if (in) dst[pos + __popc(m2 & lt)] = key;
-            }
+// Phase B of round 2 for one warp: classifies `fill` parked keys 32 at a time.  A free function
+// taking values, so that the caller's per-warp state can stay in registers.
+__device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx, const uint32_t* stage, int fill)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t lt = (1u << lane) - 1u;
+    __syncwarp();
+    for (int base = 0; base < fill; base += 32) {
+        const int i = base + lane;
+        uint32_t key = 0;
+        bool in = false;
+        if (i < fill) {
+            key = stage[i];
+            int cell, sh;
+            uint32_t low;
+            in = classify(*tb, key, cell, low, sh);
+            if (in) hist_add(ctx->cnt, ctx->lo, ctx->hi, cell, low);
         }
-        __syncwarp();
-        fill = 0;
+        const uint32_t m2 = __ballot_sync(0xffffffffu, in);
+        if (m2) {
+            unsigned long long pos = 0;
+            if (lane == 0) pos = atomicAdd(ctx->cursor, (unsigned long long)__popc(m2));
+            pos = __shfl_sync(0xffffffffu, pos, 0);
+            if (in) ctx->dst[pos + __popc(m2 & lt)] = key;
+        }
     }
+    __syncwarp();
+}
 
+struct Round2Warp {
+    const Table* tb;
+    const Round2Ctx* ctx;
+    uint32_t* stage;
+    int fill;
     uint32_t clear;
 
     __device__ __forceinline__ void one(float v, bool valid)
@@ -450,17 +454,16 @@ struct Round2Warp {
         if (bits == 0x80000000u) bits = 0u;
         const uint32_t key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
         const uint32_t blk = key >> 17;
-        park(key, valid && ((tb->coarse[blk >> 5] >> (blk & 31)) & 1u));
-    }
-
-    __device__ __forceinline__ void park(uint32_t key, bool maybe)
-    {
+        const bool maybe = valid & (bool)((tb->coarse[blk >> 5] >> (blk & 31)) & 1u);  // index is always in range
         const uint32_t m = __ballot_sync(0xffffffffu, maybe);
         if (m) {
             const int lane = threadIdx.x & 31;
             if (maybe) stage[fill + __popc(m & ((1u << lane) - 1u))] = key;
             fill += __popc(m);
-            if (fill > kStageCap - 32) drain();
+            if (fill > kStageCap - 32) {
+                round2_drain(tb, ctx, stage, fill);
+                fill = 0;
+            }
         }
     }
 };
@@ -472,8 +475,12 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
 {
     const uint32_t clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ Round2Ctx ctx;
+    __syncthreads();
+    if (threadIdx.x == 0) { ctx.cnt = cnt; ctx.lo = lo; ctx.hi = hi; ctx.dst = dst; ctx.cursor = cursor; }
+    __syncthreads();
     Round2Warp w;
-    w.tb = &tb; w.cnt = cnt; w.lo = lo; w.hi = hi; w.stage = stage; w.dst = dst; w.cursor = cursor; w.fill = 0;
+    w.tb = &tb; w.ctx = &ctx; w.stage = stage; w.fill = 0;
     w.clear = clear;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
@@ -502,7 +509,7 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
             w.one(x[u].x, ok[u]); w.one(x[u].y, ok[u]); w.one(x[u].z, ok[u]); w.one(x[u].w, ok[u]);
         }
     }
-    w.drain();
+    round2_drain(w.tb, w.ctx, w.stage, w.fill);
 }
 
 // Streams one piece of a tensor's working set: histogram of the keys inside the intervals,
@@ -650,11 +657,21 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     if (threadIdx.x == 0) S.n_keys = 0;
     if (threadIdx.x < kMaxIv) { S.ivstart[threadIdx.x] = 0; S.ivufirst[threadIdx.x] = -1; S.ivpre[threadIdx.x] = 0.0; }
     __syncthreads();
-    for (long long i = threadIdx.x; i < src_cnt; i += kSelThreads) {
-        const uint32_t key = __ldcg(buf + i);
-        if (find_new_interval(S, key) >= 0) {
-            const int pos = atomicAdd(&S.n_keys, 1);
-            if (pos < kSmallN) skeys[pos] = key;
+    for (long long i0 = threadIdx.x; i0 < src_cnt; i0 += 4 * kSelThreads) {
+        uint32_t key[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {  // issue the loads together: they come from L2
+            const long long i = i0 + (long long)u * kSelThreads;
+            ok[u] = i < src_cnt;
+            key[u] = ok[u] ? __ldcg(buf + i) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (ok[u] && find_new_interval(S, key[u]) >= 0) {
+                const int pos = atomicAdd(&S.n_keys, 1);
+                if (pos < kSmallN) skeys[pos] = key[u];
+            }
         }
     }
     __syncthreads();
