@@ -443,28 +443,19 @@ __device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx,
 
 struct Round2Warp {
     const Table* tb;
-    const Round2Ctx* ctx;
-    uint32_t* stage;
-    int fill;
+    uint32_t* stage;  // this warp's kStageCap parking slots
+    int* fillp;       // their fill counter (shared memory, bumped by the lanes that hit)
     uint32_t clear;
 
+    // Phase A for one element: no warp collective, only the lanes that pass the bitmap test do work.
     __device__ __forceinline__ void one(float v, bool valid)
     {
         uint32_t bits = __float_as_uint(v) & clear;
         if (bits == 0x80000000u) bits = 0u;
         const uint32_t key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
         const uint32_t blk = key >> 17;
-        const bool maybe = valid & (bool)((tb->coarse[blk >> 5] >> (blk & 31)) & 1u);  // index is always in range
-        const uint32_t m = __ballot_sync(0xffffffffu, maybe);
-        if (m) {
-            const int lane = threadIdx.x & 31;
-            if (maybe) stage[fill + __popc(m & ((1u << lane) - 1u))] = key;
-            fill += __popc(m);
-            if (fill > kStageCap - 32) {
-                round2_drain(tb, ctx, stage, fill);
-                fill = 0;
-            }
-        }
+        const bool maybe = valid & (bool)((tb->coarse[blk >> 5] >> (blk & 31)) & 1u);  // index always in range
+        if (maybe) stage[atomicAdd(fillp, 1)] = key;
     }
 };
 
@@ -476,11 +467,13 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
     const uint32_t clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __shared__ Round2Ctx ctx;
+    __shared__ int fills[kSelWarps];
     __syncthreads();
     if (threadIdx.x == 0) { ctx.cnt = cnt; ctx.lo = lo; ctx.hi = hi; ctx.dst = dst; ctx.cursor = cursor; }
+    if (lane == 0) fills[warp] = 0;
     __syncthreads();
     Round2Warp w;
-    w.tb = &tb; w.ctx = &ctx; w.stage = stage; w.fill = 0;
+    w.tb = &tb; w.stage = stage; w.fillp = &fills[warp];
     w.clear = clear;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
@@ -492,6 +485,7 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
         if (lane < (int)(a - pb)) { v = __ldg(grad + pb + lane); valid = true; }
         else if (lane >= 4 && lane - 4 < (int)(pe - b)) { v = __ldg(grad + b + lane - 4); valid = true; }
         w.one(v, valid);
+        __syncwarp();
     }
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     const int64_t e = b >> 2;
@@ -507,9 +501,18 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             w.one(x[u].x, ok[u]); w.one(x[u].y, ok[u]); w.one(x[u].z, ok[u]); w.one(x[u].w, ok[u]);
+            // at most 128 keys were parked since the last check, and the stage holds kStageCap = 256
+            __syncwarp();
+            const int f = *(volatile int*)w.fillp;
+            if (f > kStageCap - 128) {
+                round2_drain(w.tb, &ctx, w.stage, f);
+                if (lane == 0) *w.fillp = 0;
+                __syncwarp();
+            }
         }
     }
-    round2_drain(w.tb, w.ctx, w.stage, w.fill);
+    __syncwarp();
+    round2_drain(w.tb, &ctx, w.stage, *(volatile int*)w.fillp);
 }
 
 // Streams one piece of a tensor's working set: histogram of the keys inside the intervals,
