@@ -185,6 +185,7 @@ def run_ours(args):
     import torch
 
     import paper_2002_11082_b200 as ogq
+    from paper_2002_11082_b200.sharding import aggregate_throughput, max_over_ranks, worker_ids
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -205,7 +206,7 @@ def run_ours(args):
     bits = ogq.ogq_bits_for_levels(s)
 
     # ---- inputs: K workers' buckets, generated on the host and made resident in HBM
-    host = [make_bucket(args.workload, rank * K + k) for k in range(K)]
+    host = [make_bucket(args.workload, w) for w in worker_ids(rank, K)]
     h_off = host[0].offsets
     T, N = host[0].num_tensors, host[0].total
     off = torch.from_numpy(h_off).to(dev)
@@ -281,12 +282,7 @@ def run_ours(args):
             fn()
         b.record()
         barrier()
-        ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(a.elapsed_time(b), dist, dev)
 
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     for _ in range(warmup):
@@ -306,7 +302,7 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     ms_step = ms_total / steps
     grad_bytes = 4.0 * N * K  # fp32 gradient consumed per step and rank
-    value = world * grad_bytes / (ms_step * 1e-3) / 1e9
+    value = aggregate_throughput(grad_bytes, ms_step, world)
 
     # ---- per-stage and per-kernel times (separate instrumented passes, not part of `value`)
     ms_lqp = timed(lqp_all, steps) / steps
@@ -357,7 +353,7 @@ def run_ours(args):
         e2e_steps = min(steps, 5)
         e2e_step()
         ms_e2e = timed(e2e_step, e2e_steps) / e2e_steps
-        e2e = {"value": world * grad_bytes / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+        e2e = {"value": aggregate_throughput(grad_bytes, ms_e2e, world), "unit": UNIT,
                "h2d_bytes_per_step": int(4 * N * K), "d2h_bytes_per_step": int(4 * N),
                "ms_per_step": ms_e2e, "steps": e2e_steps}
 

@@ -1,0 +1,59 @@
+"""World-size-2 test of the cross-rank host logic of the benchmark (gloo, CPU only)."""
+import os
+import socket
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+CHILD = textwrap.dedent(
+    """
+    import os, sys
+    sys.path.insert(0, %r)
+    import torch.distributed as dist
+    from paper_2002_11082_b200.sharding import worker_ids, max_over_ranks, aggregate_throughput
+    dist.init_process_group("gloo")
+    rank, world = dist.get_rank(), dist.get_world_size()
+    ids = worker_ids(rank, 4)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, ids)
+    flat = sorted(i for g in gathered for i in g)
+    assert flat == list(range(4 * world)), flat            # disjoint and complete
+    ms = max_over_ranks(10.0 + 5.0 * rank, dist)            # rank 1 is the slow one
+    assert ms == 15.0, ms
+    assert abs(aggregate_throughput(3e9, ms, world) - 2 * 3e9 / 15e-3 / 1e9) < 1e-9
+    dist.barrier()
+    dist.destroy_process_group()
+    print("rank", rank, "ok")
+    """
+)
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def test_two_ranks_gloo():
+    port = _free_port()
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", LOCAL_RANK=str(rank),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", CHILD % ROOT], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
+    outs = [p.communicate(timeout=120)[0] for p in procs]
+    for rank, (p, out) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, out
+        assert f"rank {rank} ok" in out
+
+
+def test_single_process_defaults():
+    sys.path.insert(0, ROOT)
+    from paper_2002_11082_b200.sharding import aggregate_throughput, max_over_ranks, worker_ids
+
+    assert worker_ids(3, 8) == list(range(24, 32))
+    assert max_over_ranks(7.5) == 7.5
+    assert aggregate_throughput(1e9, 1.0, 1) == 1000.0
