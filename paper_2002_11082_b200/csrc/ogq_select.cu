@@ -32,7 +32,7 @@ constexpr int kSelW = 16;          // binades in the fine window of round 1
 constexpr int kSelM = 7;           // log2(cells per binade) in the window
 constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
 constexpr int kMidN = 131072;      // tensors up to this size are solved start to finish by one CTA of their own
-constexpr int kStageCap = 256;     // per-warp staging entries for compaction
+constexpr int kStageCap = 1024;    // per-warp staging entries for compaction
 constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
 constexpr int kSliceElems = 16384;
 constexpr int kMaxRounds = 32;
@@ -59,14 +59,17 @@ struct TState {
 #ifdef OGQ_SOLVER_TIMING
 #define OGQ_TICK(st, i) do { if (threadIdx.x == 0) (st)->tick[i] = clock64(); } while (0)
 // per-CTA wall-clock record of the round-1 and round-2 kernels: start, end, time in solver passes, passes
-__device__ unsigned long long g_dbg_cta[2][4096][4];
+__device__ unsigned long long g_dbg_cta[2][4096][8];
 __device__ __forceinline__ unsigned long long dbg_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define OGQ_CTA_BEGIN(k) unsigned long long dbg_t0 = dbg_now(), dbg_solver = 0, dbg_passes = 0; const int dbg_k = (k);
+#define OGQ_CTA_BEGIN(k) unsigned long long dbg_t0 = dbg_now(), dbg_solver = 0, dbg_passes = 0, dbg_ph[4] = {0, 0, 0, 0}, dbg_last = dbg_t0; const int dbg_k = (k);
+// adds the time since the previous mark to phase i (0 setup, 1 streaming, 2 flush, 3 combine / arrive)
+#define OGQ_CTA_PHASE(i) do { const unsigned long long n_ = dbg_now(); dbg_ph[i] += n_ - dbg_last; dbg_last = n_; } while (0)
 #define OGQ_CTA_SOLVER(expr) do { unsigned long long a_ = dbg_now(); expr; dbg_solver += dbg_now() - a_; ++dbg_passes; } while (0)
-#define OGQ_CTA_END() do { if (threadIdx.x == 0 && blockIdx.x < 4096) { g_dbg_cta[dbg_k][blockIdx.x][0] = dbg_t0; g_dbg_cta[dbg_k][blockIdx.x][1] = dbg_now(); g_dbg_cta[dbg_k][blockIdx.x][2] = dbg_solver; g_dbg_cta[dbg_k][blockIdx.x][3] = dbg_passes; } } while (0)
+#define OGQ_CTA_END() do { if (threadIdx.x == 0 && blockIdx.x < 4096) { g_dbg_cta[dbg_k][blockIdx.x][0] = dbg_t0; g_dbg_cta[dbg_k][blockIdx.x][1] = dbg_now(); g_dbg_cta[dbg_k][blockIdx.x][2] = dbg_solver; g_dbg_cta[dbg_k][blockIdx.x][3] = dbg_passes; for (int q_ = 0; q_ < 4; ++q_) g_dbg_cta[dbg_k][blockIdx.x][4 + q_] = dbg_ph[q_]; } } while (0)
 #else
 #define OGQ_TICK(st, i) do { } while (0)
 #define OGQ_CTA_BEGIN(k)
+#define OGQ_CTA_PHASE(i) do { } while (0)
 #define OGQ_CTA_SOLVER(expr) do { expr; } while (0)
 #define OGQ_CTA_END() do { } while (0)
 #endif
@@ -185,18 +188,6 @@ __device__ __forceinline__ void round1_cell(uint32_t bits, int lo_e, bool magnit
 }
 
 __device__ __forceinline__ uint32_t key_to_bits(uint32_t k) { return (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k; }
-
-// Marks every block of 2^17 keys that intersects one of the table's intervals (called by all threads).
-__device__ __forceinline__ void build_prefilter(Table& tb)
-{
-    for (int i = threadIdx.x; i < 1024; i += kSelThreads) tb.coarse[i] = 0u;
-    __syncthreads();
-    if ((int)threadIdx.x < tb.m) {
-        const uint32_t ba = tb.klo[threadIdx.x] >> 17, bb = tb.khi[threadIdx.x] >> 17;
-        for (uint32_t b = ba; b <= bb; ++b) atomicOr(&tb.coarse[b >> 5], 1u << (b & 31));
-    }
-    __syncthreads();
-}
 
 __device__ __forceinline__ bool classify(const Table& tb, uint32_t key, int& cell, uint32_t& low, int& sh)
 {
@@ -333,50 +324,57 @@ __device__ __forceinline__ void visit_plain(const float* __restrict__ grad, int6
     }
 }
 
-// Round 1 over grad[pb, pe): per element the round-1 cell (count and low-key-bit sum with carry) and
-// the running min / max key.  Non-finite values show up as extreme keys afterwards.
+// Round 1 over grad[pb, pe).  Per element two shared atomics without a return value: the cell's
+// count and the sum of its low key bits.  Inside the fine window the low bits are below 2^16 and a
+// CTA flushes its cells at least every kR1MaxPiece = 2^16 elements, so that sum cannot overflow 32
+// bits; only the rare values outside the window (23 low bits) go through the carry word.  Min and
+// max are tracked as floats; -0 is folded into +0 by adding +0 first.
+constexpr int64_t kR1MaxPiece = (int64_t)1 << 16;
+
+template <bool MAG>
 struct Round1Body {
-    uint32_t lo23, clear;
-    int lo_e, base;
-    uint32_t* hist;  // counts at [0, kCells), low sums at [kCells, 2 kCells), carries above
-    uint32_t mn, mx;
+    uint32_t lo23;
+    int lo_e;
+    uint32_t* cnt;  // counts, already offset to the first non-negative magnitude cell; low sums at
+                    // + kCells, their carries at + 2 kCells
+    float mn, mx;
+    uint32_t nonfinite;
 
     __device__ __forceinline__ void operator()(float v)
     {
-        uint32_t bits = __float_as_uint(v) & clear;
-        if (bits == 0x80000000u) bits = 0u;
-        const int sgn = (int)bits >> 31;  // 0 or -1
-        const uint32_t mag = bits & 0x7fffffffu;
+        v = (MAG ? fabsf(v) : v) + 0.0f;
+        const uint32_t bits = __float_as_uint(v);
+        const int sgn = MAG ? 0 : ((int)bits >> 31);  // 0 or -1
+        const uint32_t mag = MAG ? bits : (bits & 0x7fffffffu);
         const uint32_t rel = mag - lo23;
-        int mi = lo_e + (int)(rel >> (23 - kSelM));
-        uint32_t mask = (1u << (23 - kSelM)) - 1u;
-        if (rel >= ((uint32_t)kSelW << 23)) {  // outside the fine window: one cell per binade
+        mn = fminf(mn, v);
+        mx = fmaxf(mx, v);
+        if (rel < ((uint32_t)kSelW << 23)) {
+            uint32_t* c = cnt + ((lo_e + (int)(rel >> (23 - kSelM))) ^ sgn);
+            atomicAdd(c, 1u);
+            atomicAdd(c + kCells, (mag ^ (uint32_t)sgn) & ((1u << (23 - kSelM)) - 1u));
+        } else {  // outside the fine window: one cell per binade
             const int e = (int)(mag >> 23);
-            mi = (e < lo_e) ? e : e - kSelW + (kSelW << kSelM);
-            mask = 0x7fffffu;
+            const int mi = (e < lo_e) ? e : e - kSelW + (kSelW << kSelM);
+            if (e == 255) nonfinite = 1u;  // the window never reaches binade 255
+            uint32_t* c = cnt + (mi ^ sgn);
+            const uint32_t low = (mag ^ (uint32_t)sgn) & 0x7fffffu;
+            atomicAdd(c, 1u);
+            const uint32_t old = atomicAdd(c + kCells, low);
+            if (old + low < old) atomicAdd(c + 2 * kCells, 1u);
         }
-        const int cell = base + (mi ^ sgn);
-        const uint32_t lowkey = (mag ^ (uint32_t)sgn) & mask;
-        const uint32_t key = bits ^ ((uint32_t)sgn | 0x80000000u);
-        mn = key < mn ? key : mn;
-        mx = key > mx ? key : mx;
-        atomicAdd(hist + cell, 1u);
-        const uint32_t old = atomicAdd(hist + kCells + cell, lowkey);
-        if (old + lowkey < old) atomicAdd(hist + 2 * kCells + cell, 1u);
     }
 };
 
-__device__ __forceinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe,
-                                              bool magnitude_only, int lo_e, uint32_t* cnt, uint32_t* lo,
-                                              uint32_t* hi, uint32_t& kmin, uint32_t& kmax)
+template <bool MAG>
+__device__ __forceinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe, int lo_e,
+                                              uint32_t* hist, float& vmin, float& vmax, uint32_t& nonfinite)
 {
-    Round1Body f;
+    Round1Body<MAG> f;
     f.lo23 = (uint32_t)lo_e << 23;
-    f.clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
     f.lo_e = lo_e;
-    f.base = magnitude_only ? 0 : kRound1Mag;
-    f.hist = cnt;
-    f.mn = kmin; f.mx = kmax;
+    f.cnt = hist + (MAG ? 0 : kRound1Mag);
+    f.mn = vmin; f.mx = vmax; f.nonfinite = nonfinite;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
     int64_t b = pe & ~(int64_t)3;
@@ -398,33 +396,37 @@ __device__ __forceinline__ void stream_round1(const float* __restrict__ grad, in
         const float4 x = __ldg(g4 + i);
         f(x.x); f(x.y); f(x.z); f(x.w);
     }
-    kmin = f.mn;
-    kmax = f.mx;
+    vmin = f.mn; vmax = f.mx; nonfinite = f.nonfinite;
 }
 
-// Round 2 over grad[pb, pe).  Phase A: a one-bit-per-2^17-keys test rejects almost every element;
-// keys that pass are parked in the warp's stage (ballot + popc, no classification yet).  Phase B,
-// whenever the stage fills up: the parked keys are classified exactly 32 at a time, so that the
-// expensive part runs with all lanes busy; keys inside an interval are histogrammed and copied out.
+// Round 2 over grad[pb, pe).  Phase A: a one-bit-per-2^17-bit-patterns test on the raw fp32 bits
+// rejects almost every element; values that pass are parked in the warp's stage (no classification
+// yet).  Phase B, whenever the stage fills up: the parked values are turned into keys and classified
+// exactly 32 at a time, so that the expensive part runs with all lanes busy; keys inside an interval
+// are histogrammed and copied out.
 struct Round2Ctx {  // per-CTA constants of round 2, kept in shared memory to spare registers
     uint32_t *cnt, *lo, *hi;
     uint32_t* dst;
     unsigned long long* cursor;
+    uint32_t clear;  // 0x7fffffff when only magnitudes count
 };
 
-// Phase B of round 2 for one warp: classifies `fill` parked keys 32 at a time.  A free function
+// Phase B of round 2 for one warp: classifies `fill` parked values 32 at a time.  A free function
 // taking values, so that the caller's per-warp state can stay in registers.
 __device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx, const uint32_t* stage, int fill)
 {
     const int lane = threadIdx.x & 31;
     const uint32_t lt = (1u << lane) - 1u;
+    const uint32_t clear = ctx->clear;
     __syncwarp();
     for (int base = 0; base < fill; base += 32) {
         const int i = base + lane;
         uint32_t key = 0;
         bool in = false;
         if (i < fill) {
-            key = stage[i];
+            uint32_t bits = stage[i] & clear;
+            if (bits == 0x80000000u) bits = 0u;
+            key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
             int cell, sh;
             uint32_t low;
             in = classify(*tb, key, cell, low, sh);
@@ -441,21 +443,40 @@ __device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx,
     __syncwarp();
 }
 
+// Marks, in the space of raw fp32 bit patterns, every block of 2^17 patterns that can hold a value
+// whose key lies in one of the table's intervals (called by all threads).  A block of 2^17 aligned
+// keys is a block of 2^17 aligned patterns; -0 shares the block of the smallest negative values, and
+// with magnitude_only both signs of a pattern are marked.
+__device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
+{
+    for (int i = threadIdx.x; i < 1024; i += kSelThreads) tb.coarse[i] = 0u;
+    __syncthreads();
+    if ((int)threadIdx.x < tb.m) {
+        const uint32_t ba = tb.klo[threadIdx.x] >> 17, bb = tb.khi[threadIdx.x] >> 17;
+        for (uint32_t b = ba; b <= bb; ++b) {
+            const uint32_t pblk = (b & 0x4000u) ? (b ^ 0x4000u) : (~b & 0x7fffu);
+            atomicOr(&tb.coarse[pblk >> 5], 1u << (pblk & 31));
+            if (magnitude_only || pblk == 0u) {
+                const uint32_t twin = pblk ^ 0x4000u;
+                atomicOr(&tb.coarse[twin >> 5], 1u << (twin & 31));
+            }
+        }
+    }
+    __syncthreads();
+}
+
 struct Round2Warp {
-    const Table* tb;
-    uint32_t* stage;  // this warp's kStageCap parking slots
-    int* fillp;       // their fill counter (shared memory, bumped by the lanes that hit)
-    uint32_t clear;
+    const uint32_t* coarse;  // the table's prefilter bitmap
+    uint32_t* stage;         // this warp's kStageCap parking slots
+    int* fillp;              // their fill counter (shared memory, bumped by the lanes that hit)
 
     // Phase A for one element: no warp collective, only the lanes that pass the bitmap test do work.
-    __device__ __forceinline__ void one(float v, bool valid)
+    __device__ __forceinline__ void one(float v)
     {
-        uint32_t bits = __float_as_uint(v) & clear;
-        if (bits == 0x80000000u) bits = 0u;
-        const uint32_t key = bits ^ ((uint32_t)((int)bits >> 31) | 0x80000000u);
-        const uint32_t blk = key >> 17;
-        const bool maybe = valid & (bool)((tb->coarse[blk >> 5] >> (blk & 31)) & 1u);  // index always in range
-        if (maybe) stage[atomicAdd(fillp, 1)] = key;
+        const uint32_t bits = __float_as_uint(v);
+        const uint32_t word = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(coarse) +
+                                                                 ((bits >> 20) & 0xffcu));
+        if (__funnelshift_r(word, 0u, bits >> 17) & 1u) stage[atomicAdd(fillp, 1)] = bits;
     }
 };
 
@@ -464,55 +485,61 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
                                               uint32_t* hi, uint32_t* stage, uint32_t* dst,
                                               unsigned long long* cursor)
 {
-    const uint32_t clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __shared__ Round2Ctx ctx;
     __shared__ int fills[kSelWarps];
     __syncthreads();
-    if (threadIdx.x == 0) { ctx.cnt = cnt; ctx.lo = lo; ctx.hi = hi; ctx.dst = dst; ctx.cursor = cursor; }
+    if (threadIdx.x == 0) {
+        ctx.cnt = cnt; ctx.lo = lo; ctx.hi = hi; ctx.dst = dst; ctx.cursor = cursor;
+        ctx.clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
+    }
     if (lane == 0) fills[warp] = 0;
     __syncthreads();
     Round2Warp w;
-    w.tb = &tb; w.stage = stage; w.fillp = &fills[warp];
-    w.clear = clear;
+    w.coarse = tb.coarse; w.stage = stage; w.fillp = &fills[warp];
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
     int64_t b = pe & ~(int64_t)3;
     if (b < a) b = a;
     if (warp == 0) {  // ragged head and tail, one element per lane
-        float v = 0.f;
-        bool valid = false;
-        if (lane < (int)(a - pb)) { v = __ldg(grad + pb + lane); valid = true; }
-        else if (lane >= 4 && lane - 4 < (int)(pe - b)) { v = __ldg(grad + b + lane - 4); valid = true; }
-        w.one(v, valid);
+        if (lane < (int)(a - pb)) w.one(__ldg(grad + pb + lane));
+        else if (lane >= 4 && lane - 4 < (int)(pe - b)) w.one(__ldg(grad + b + lane - 4));
         __syncwarp();
     }
+    // at most 32 * 16 = 512 values are parked between two checks, and the stage holds kStageCap = 1024
+    auto check = [&]() {
+        __syncwarp();
+        const int f = *(volatile int*)w.fillp;
+        if (f > kStageCap - 512) {
+            round2_drain(&tb, &ctx, w.stage, f);
+            if (lane == 0) *w.fillp = 0;
+            __syncwarp();
+        }
+    };
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     const int64_t e = b >> 2;
-    for (int64_t i0 = (a >> 2) + warp * 32; i0 < e; i0 += 4 * kSelThreads) {  // trip count is warp-uniform
+    int64_t i0 = (a >> 2) + warp * 32;  // the trip counts below are warp-uniform
+    for (; i0 + 3 * kSelThreads + 32 <= e; i0 += 4 * kSelThreads) {
         float4 x[4];
-        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i0 + lane + u * kSelThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { w.one(x[u].x); w.one(x[u].y); w.one(x[u].z); w.one(x[u].w); }
+        check();
+    }
+    if (i0 < e) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int64_t i = i0 + lane + (int64_t)u * kSelThreads;
-            ok[u] = i < e;
-            x[u] = ok[u] ? __ldg(g4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            w.one(x[u].x, ok[u]); w.one(x[u].y, ok[u]); w.one(x[u].z, ok[u]); w.one(x[u].w, ok[u]);
-            // at most 128 keys were parked since the last check, and the stage holds kStageCap = 256
-            __syncwarp();
-            const int f = *(volatile int*)w.fillp;
-            if (f > kStageCap - 128) {
-                round2_drain(w.tb, &ctx, w.stage, f);
-                if (lane == 0) *w.fillp = 0;
-                __syncwarp();
+            if (i < e) {
+                const float4 x = __ldg(g4 + i);
+                w.one(x.x); w.one(x.y); w.one(x.z); w.one(x.w);
             }
         }
+        check();
     }
     __syncwarp();
-    round2_drain(w.tb, &ctx, w.stage, *(volatile int*)w.fillp);
+    round2_drain(&tb, &ctx, w.stage, *(volatile int*)w.fillp);
 }
 
 // Streams one piece of a tensor's working set: histogram of the keys inside the intervals,
@@ -1410,7 +1437,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
     __shared__ SolverShared S;
     __shared__ Interval r1iv[kMaxIv];
     __shared__ int sh_i[kSelWarps];
-    __shared__ uint32_t sh_u[2 * kSelWarps];
     __shared__ int sh_last;
     const bool pb = A.scheme == OGQ_BINGRAD_PB;
     const int nl = pb ? 2 : A.s;
@@ -1423,55 +1449,70 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
     auto do_round1 = [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_, bool alone) -> bool {
         const int64_t n = tend - tbeg;
         TState* st = A.ws.st + t;
-        // anchor of the fine window: largest binade among strided samples, plus two
-        int e = 0;
+        // anchor of the fine window: largest binade among strided samples, plus two (every CTA of the
+        // tensor samples the same elements and so arrives at the same window)
+        int hi_e;
         {
             const int64_t idx = tbeg + (int64_t)threadIdx.x * n / kSelThreads;
-            e = (int)((__float_as_uint(__ldg(A.grad + idx)) >> 23) & 255u);
+            int e = (int)((__float_as_uint(__ldg(A.grad + idx)) >> 23) & 255u);
             if (e == 255) e = 0;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) { const int x = __shfl_xor_sync(0xffffffffu, e, o); e = x > e ? x : e; }
-        }
-        __syncthreads();
-        if ((threadIdx.x & 31) == 0) sh_i[threadIdx.x >> 5] = e;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int mx = 0;
-            for (int w = 0; w < kSelWarps; ++w) mx = sh_i[w] > mx ? sh_i[w] : mx;
-            int hi_e = mx + 2;
+            e = __reduce_max_sync(0xffffffffu, e);
+            __syncthreads();  // earlier readers of sh_i are done
+            if ((threadIdx.x & 31) == 0) sh_i[threadIdx.x >> 5] = e;
+            __syncthreads();
+            hi_e = __reduce_max_sync(0xffffffffu, sh_i[threadIdx.x & 31]) + 2;
             if (hi_e < kSelW) hi_e = kSelW;
-            if (hi_e > 256) hi_e = 256;
-            const int m = round1_intervals(hi_e, pb, r1iv);
-            table_from_intervals(tb, r1iv, m);
-            tb.lo_e = hi_e - kSelW;
+            if (hi_e > 255) hi_e = 255;  // binade 255 (Inf / NaN) always stays outside the fine window
         }
+        const int lo_e = hi_e - kSelW;
+        const int ncells = pb ? kRound1Mag : kRound1Cells;
+        uint32_t* gcnt = A.ws.gcnt + (size_t)t * kCells;
+        unsigned long long* glsum = A.ws.glsum + (size_t)t * kCells;
+        float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
+        uint32_t nf = 0u;
+        zero_hist(hist, ncells);
         __syncthreads();
-        zero_hist(hist, tb.ncells);
+        OGQ_CTA_PHASE(0);
+        if (pb) stream_round1<true>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf);
+        else stream_round1<false>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf);
         __syncthreads();
-        uint32_t kmin = 0xffffffffu, kmax = 0u, nf = 0u;
-        stream_round1(A.grad, pb_, pe_, pb, tb.lo_e, hist, hist + kCells, hist + 2 * kCells, kmin, kmax);
-        nf = (kmax >= 0xff800000u || kmin <= 0x007fffffu) ? 1u : 0u;  // Inf / NaN keys lie beyond these
-        // combine min / max / non-finite over the CTA, then one atomic each
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const uint32_t a = __shfl_xor_sync(0xffffffffu, kmin, o), b = __shfl_xor_sync(0xffffffffu, kmax, o);
-            kmin = a < kmin ? a : kmin;
-            kmax = b > kmax ? b : kmax;
-            nf |= __shfl_xor_sync(0xffffffffu, nf, o);
+        OGQ_CTA_PHASE(1);
+        // The low sums of the window's cells are 32 bits wide without a carry: exact as long as no such
+        // cell took more than 2^16 values.  Otherwise (heavily repeated values) the piece is redone in
+        // parts of kR1MaxPiece elements, flushed one by one.
+        bool crowded = false;
+        if (pe_ - pb_ > kR1MaxPiece) {
+            const int base = pb ? 0 : kRound1Mag;
+            for (int i = threadIdx.x; i < ncells; i += kSelThreads) {
+                const int mi = (i >= base) ? i - base : base - 1 - i;
+                crowded |= hist[i] > (uint32_t)kR1MaxPiece && mi >= lo_e && mi < lo_e + (kSelW << kSelM);
+            }
         }
-        __syncthreads();
-        if ((threadIdx.x & 31) == 0) {
-            sh_u[threadIdx.x >> 5] = kmin;
-            sh_u[kSelWarps + (threadIdx.x >> 5)] = kmax;
-            if (nf) atomicOr(&st->nonfinite, 1u);
+        if (__syncthreads_or(crowded)) {
+            for (int64_t q = pb_; q < pe_; q += kR1MaxPiece) {
+                const int64_t qe = (q + kR1MaxPiece < pe_) ? q + kR1MaxPiece : pe_;
+                zero_hist(hist, ncells);
+                __syncthreads();
+                if (pb) stream_round1<true>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf);
+                else stream_round1<false>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf);
+                __syncthreads();
+                flush_hist(hist, ncells, gcnt, glsum);
+                __syncthreads();
+            }
+        } else {
+            flush_hist(hist, ncells, gcnt, glsum);
         }
-        __syncthreads();
-        flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
-        if (threadIdx.x == 0) {
-            uint32_t mn = 0xffffffffu, mx = 0u;
-            for (int w = 0; w < kSelWarps; ++w) { mn = sh_u[w] < mn ? sh_u[w] : mn; mx = sh_u[kSelWarps + w] > mx ? sh_u[kSelWarps + w] : mx; }
-            atomicMax(&st->kmin_inv, ~mn);
-            atomicMax(&st->kmax, mx);
+        OGQ_CTA_PHASE(2);
+        // min / max / non-finite: one atomic per warp
+        {
+            const uint32_t kmin = __reduce_min_sync(0xffffffffu, float_to_key(vmin));  // +Inf / -Inf when the
+            const uint32_t kmax = __reduce_max_sync(0xffffffffu, float_to_key(vmax));  // thread saw nothing
+            const bool anynf = __any_sync(0xffffffffu, nf != 0u);
+            if ((threadIdx.x & 31) == 0) {
+                atomicMax(&st->kmin_inv, ~kmin);
+                atomicMax(&st->kmax, kmax);
+                if (anynf) atomicOr(&st->nonfinite, 1u);
+            }
         }
         __threadfence();
         __syncthreads();
@@ -1482,6 +1523,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
                 sh_last = (prev == (unsigned)(c1 - c0));
             }
             __syncthreads();
+            OGQ_CTA_PHASE(3);
             if (!sh_last) return false;
             __threadfence();
         }
@@ -1490,9 +1532,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
         if (threadIdx.x == 0) {
             st->n = n;
             st->round = 1;
-            st->hi_e = tb.lo_e + kSelW;
-            st->m = tb.m;
-            for (int j = 0; j < tb.m; ++j) st->iv[j] = r1iv[j];
+            st->hi_e = hi_e;
+            const int m = round1_intervals(hi_e, pb, r1iv);
+            st->m = m;
+            for (int j = 0; j < m; ++j) st->iv[j] = r1iv[j];
             int stb = 0;
             const uint32_t kmn = ~__ldcg(&st->kmin_inv), kmx = __ldcg(&st->kmax);
             if (__ldcg(&st->nonfinite)) stb |= OGQ_ST_NONFINITE;
@@ -1538,7 +1581,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
                 tb.lo_e = st->hi_e - kSelW;
             }
             __syncthreads();
-            build_prefilter(tb);
+            build_prefilter(tb, pb);
             zero_hist(hist, tb.ncells);
             __syncthreads();
             stream_round2(A.grad, tbeg, tend, pb, tb, hist, hist + kCells, hist + 2 * kCells,
@@ -1588,7 +1631,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round2(SelArgs A)
             tb.lo_e = st->hi_e - kSelW;
         }
         __syncthreads();
-        build_prefilter(tb);
+        build_prefilter(tb, pb);
         zero_hist(hist, tb.ncells);
         __syncthreads();
         stream_round2(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells,
@@ -1665,9 +1708,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round3(SelArgs A)
 }
 
 #ifdef OGQ_SOLVER_TIMING
-extern "C" int ogq_debug_dump_ctas(unsigned long long* h_out /*[2][4096][4]*/)
+extern "C" int ogq_debug_dump_ctas(unsigned long long* h_out /*[2][4096][8]*/)
 {
-    return cudaMemcpyFromSymbol(h_out, g_dbg_cta, sizeof(unsigned long long) * 2 * 4096 * 4) == cudaSuccess ? 0 : -1;
+    return cudaMemcpyFromSymbol(h_out, g_dbg_cta, sizeof(unsigned long long) * 2 * 4096 * 8) == cudaSuccess ? 0 : -1;
 }
 extern "C" int ogq_debug_dump_ticks(const void* d_ws, int T, long long* h_out /*[T][16]*/, int* h_round, long long* h_n)
 {

@@ -174,3 +174,22 @@ def test_flat_sweep_tensor(log2n):
     lv, th, _ = db.levels_bingrad(ogq.OGQ_BINGRAD_B, 0)
     w_lv, w_th, _ = oracle.bucket_levels_bingrad(b.values, b.offsets, oracle.B, 0)
     assert levels_close(lv[0], w_lv[0])
+
+
+def test_flat_tensor_with_crowded_cells():
+    """A tensor large enough that every CTA streams more than 2^16 elements, 90 % of them one
+    repeated non-zero value: the levels still satisfy the optimal condition exactly."""
+    r = np.random.Generator(np.random.PCG64(23))
+    n = 48_000_000
+    v = wl.gaussian(r, n, 1e-3)
+    v[r.random(n) < 0.9] = np.float32(2.5e-3)
+    off = np.array([0, n], np.int64)
+    db = DeviceBucket(v, off)
+    for s in (3, 9):
+        lv, st = db.levels_orq(s)
+        assert st[0] == 0
+        check_orq_levels_by_condition(v, lv[0])
+    v[12_345_678] = np.nan
+    db = DeviceBucket(v, off)
+    lv, st = db.levels_orq(9)
+    assert st[0] & ogq.OGQ_ST_NONFINITE

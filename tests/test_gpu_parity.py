@@ -151,6 +151,32 @@ def test_levels_bingrad_pb(bucket_fn):
     assert np.array_equal(lv, lv2)
 
 
+def crowded_bucket(seed=17):
+    """Tensors in which one non-zero value is repeated more than 2^16 times inside the piece a single
+    CTA streams, next to ordinary data (the histogram's 32-bit partial sums must not wrap)."""
+    r = rng(seed)
+    parts = []
+    for n, rep, frac in ((131072, 0.37, 0.95), (120000, -1.5e-3, 0.9), (131072, 2.5e-3, 0.7)):
+        v = wl.gaussian(r, n, 1e-3)
+        v[r.random(n) < frac] = np.float32(rep)
+        parts.append(v)
+    return wl.Bucket(np.concatenate(parts), wl.offsets_from_sizes([p.size for p in parts]), ["a", "b", "c"])
+
+
+@pytest.mark.parametrize("s", [3, 9])
+def test_levels_crowded_cells(s):
+    b = crowded_bucket()
+    db = DeviceBucket(b.values, b.offsets)
+    lv, st = db.levels_orq(s)
+    w_lv, w_st = oracle.bucket_levels_orq(b.values, b.offsets, s)
+    assert np.array_equal(st, w_st)
+    assert np.array_equal(lv, w_lv)
+    lv, _, st = db.levels_bingrad(ogq.OGQ_BINGRAD_PB)
+    w_lv, _, w_st = oracle.bucket_levels_bingrad(b.values, b.offsets, oracle.PB)
+    assert np.array_equal(st, w_st)
+    assert_levels_close(lv, w_lv, "pb")
+
+
 def test_levels_nonfinite_is_flagged_not_trapped():
     vals = np.concatenate([wl.laplace(rng(1), 10000, 1e-3), wl.laplace(rng(2), 3000, 1e-3)])
     vals[77] = np.nan
