@@ -51,11 +51,12 @@ template <int BITS, bool THRESHOLD>
 __global__ void __launch_bounds__(kThreads)
 k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off, int T, int64_t total,
                 int64_t chunk, int s, const float* __restrict__ levels, const float* __restrict__ thresh,
-                uint32_t seed_lo, uint32_t seed_hi, uint32_t stream_id,
+                const __grid_constant__ PhiloxKeys keys, uint32_t stream_id,
                 const int64_t* __restrict__ packed_off, uint32_t* __restrict__ packed)
 {
     __shared__ float sh_lv[kMaxLevels];
     __shared__ float sh_w[kMaxLevels];
+    __shared__ float2 sh_tab[kMaxLevels];  // {level k, width of the segment above it}
 
     const int64_t lo = (int64_t)blockIdx.x * chunk;
     const int64_t hi = (lo + chunk < total) ? lo + chunk : total;
@@ -75,6 +76,8 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                 const float prv = threadIdx.x > 0 ? __ldg(levels + (int64_t)t * s + threadIdx.x - 1) : cur;
                 sh_lv[threadIdx.x] = cur;
                 sh_w[threadIdx.x] = __fsub_rn(cur, prv);  // width of the segment below level k
+                const float nxt = (int)threadIdx.x + 1 < s ? __ldg(levels + (int64_t)t * s + threadIdx.x + 1) : cur;
+                sh_tab[threadIdx.x] = make_float2(cur, __fsub_rn(nxt, cur));
             }
             __syncthreads();
         }
@@ -83,7 +86,61 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
         const bool aligned = (tb & 3) == 0;
         const float* base = grad + tb;
 
-        for (int64_t g = g_beg + warp; g < g_end; g += kWarps) {
+        // Fast path: groups that lie wholly inside the tensor, 128-bit loads, two groups in flight
+        // per warp, no bounds checks.  The generic loop below takes what is left (the last, partial
+        // group; everything when the tensor does not start on a 16-byte boundary).
+        int64_t g_rest = g_beg;
+        if (!THRESHOLD && (BITS == 1 || BITS == 2 || BITS == 4) && aligned) {
+            const int64_t g_full = (n >> 7) < g_end ? (n >> 7) : g_end;
+            if (g_full > g_beg) {
+                g_rest = g_full;
+                constexpr int L = 8 / BITS;
+                const int ng = (int)(g_full - g_beg);
+                const float4* src = reinterpret_cast<const float4*>(base + (g_beg << 7)) + lane;
+                uint32_t* dstw = out + g_beg * (4 * BITS) + lane / L;
+                const uint64_t q0 = ((uint64_t)g_beg << 5) + (uint64_t)lane;
+                const bool writer = (lane & (L - 1)) == 0;
+                auto code4 = [&](const float4 v, int gl) -> uint32_t {
+                    const uint64_t q = q0 + ((uint64_t)(uint32_t)gl << 5);
+                    const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)t, stream_id, keys);
+                    const float xs[4] = {v.x, v.y, v.z, v.w};
+                    const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+                    uint32_t bits4 = 0u;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        int idx = 0;
+#pragma unroll
+                        for (int step = (BITS >= 2) ? (1 << (BITS - 2)) : 0; step >= 1; step >>= 1)
+                            if (sh_tab[idx + step].x <= xs[j]) idx += step;
+                        const float2 e = sh_tab[idx];
+                        const float lhs = __fmul_rn((float)(rw[j] >> 8), e.y);
+                        const float rhs = __fmul_rn(__fsub_rn(xs[j], e.x), 16777216.0f);
+                        bits4 |= ((uint32_t)idx + ((lhs < rhs) ? 1u : 0u)) << (j * BITS);
+                    }
+                    return assemble_words<BITS>(bits4, lane);
+                };
+                // software pipeline: the loads of the next two groups are issued before the current two
+                // are quantized
+                int gl = warp;
+                const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 va = (gl < ng) ? __ldg(src + (size_t)gl * 32) : zero4;
+                float4 vb = (gl + kWarps < ng) ? __ldg(src + (size_t)(gl + kWarps) * 32) : zero4;
+                for (; gl < ng; gl += 2 * kWarps) {
+                    const int gn = gl + 2 * kWarps;
+                    const float4 na = (gn < ng) ? __ldg(src + (size_t)gn * 32) : zero4;
+                    const float4 nb = (gn + kWarps < ng) ? __ldg(src + (size_t)(gn + kWarps) * 32) : zero4;
+                    const uint32_t wa = code4(va, gl);
+                    if (writer) dstw[(size_t)gl * (4 * BITS)] = wa;
+                    if (gl + kWarps < ng) {
+                        const uint32_t wb = code4(vb, gl + kWarps);
+                        if (writer) dstw[(size_t)(gl + kWarps) * (4 * BITS)] = wb;
+                    }
+                    va = na; vb = nb;
+                }
+            }
+        }
+
+        for (int64_t g = g_rest + warp; g < g_end; g += kWarps) {
             const int64_t i0 = (g << 7) + 4 * lane;
             float x[4];
             if (aligned && i0 + 3 < n) {
@@ -99,8 +156,7 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                 for (int j = 0; j < 4; ++j) c[j] = (x[j] >= b0) ? 1u : 0u;
             } else {
                 const uint64_t q = (uint64_t)i0 >> 2;
-                const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)t, stream_id,
-                                              seed_lo, seed_hi);
+                const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)t, stream_id, keys);
                 const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -159,9 +215,11 @@ k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* _
         const int64_t g_beg = (pb - tb + 127) >> 7, g_end = (pe - tb + 127) >> 7;
         if (g_beg >= g_end) return;
         __syncthreads();
-        for (int i = threadIdx.x; i < K * s; i += kThreads) {
-            const int k = i / s, q = i - k * s;
-            sh_lv[k][q] = __ldg(levels_k[k] + (int64_t)t * s + q);
+        // every code a BITS-bit field can hold gets an entry: codes above s - 1 (never produced by the
+        // quantizer) read the top level, so the inner loops need no clamp
+        for (int i = threadIdx.x; i < K * 32; i += kThreads) {
+            const int k = i >> 5, q = i & 31;
+            sh_lv[k][q] = __ldg(levels_k[k] + (int64_t)t * s + (q < s ? q : s - 1));
         }
         const int64_t pofs = __ldg(packed_off + t);
         if (threadIdx.x < K) sh_pk[threadIdx.x] = packed_k[threadIdx.x] + pofs;
@@ -170,7 +228,55 @@ k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* _
         const bool aligned = (tb & 3) == 0;
         float* dst = outp + tb;
 
-        for (int64_t g = g_beg + warp; g < g_end; g += kWarps) {
+        // Fast path (1, 2 or 4 bits per code): groups wholly inside the tensor, eight workers' words in
+        // flight per lane, level rows addressed with compile-time offsets.  All lanes of a warp read the
+        // same few level entries, so the shared-memory loads are broadcasts.
+        int64_t g_rest = g_beg;
+        if ((BITS == 1 || BITS == 2 || BITS == 4) && aligned) {
+            const int64_t g_full = (n >> 7) < g_end ? (n >> 7) : g_end;
+            if (g_full > g_beg) {
+                g_rest = g_full;
+                constexpr int L = 8 / BITS;                       // lanes per packed word
+                const int shift = (lane & (L - 1)) * 4 * BITS;    // this lane's 4 codes inside its word
+                const int64_t w0 = g_beg * (4 * BITS) + lane / L;
+                float4* dst4 = reinterpret_cast<float4*>(dst + (g_beg << 7)) + lane;
+                const int ng = (int)(g_full - g_beg);
+                const char* rows = reinterpret_cast<const char*>(&sh_lv[0][0]);
+                constexpr int kRow = (kMaxLevels + 1) * (int)sizeof(float);
+                for (int gl = warp; gl < ng; gl += kWarps) {
+                    const int64_t wi = w0 + (int64_t)gl * (4 * BITS);
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                    int k0 = 0;
+                    for (; k0 + 8 <= K; k0 += 8) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) w[u] = __ldg(sh_pk[k0 + u] + wi);
+                        const char* r0 = rows + k0 * kRow;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const uint32_t f = (w[u] >> shift) << 2;  // byte offsets of the 4 codes
+                            const char* r = r0 + u * kRow;
+                            a0 = __fadd_rn(a0, *reinterpret_cast<const float*>(r + (f & (kMask1 << 2))));
+                            a1 = __fadd_rn(a1, *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2))));
+                            a2 = __fadd_rn(a2, *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2))));
+                            a3 = __fadd_rn(a3, *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2))));
+                        }
+                    }
+                    for (; k0 < K; ++k0) {
+                        const uint32_t f = (__ldg(sh_pk[k0] + wi) >> shift) << 2;
+                        const char* r = rows + k0 * kRow;
+                        a0 = __fadd_rn(a0, *reinterpret_cast<const float*>(r + (f & (kMask1 << 2))));
+                        a1 = __fadd_rn(a1, *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2))));
+                        a2 = __fadd_rn(a2, *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2))));
+                        a3 = __fadd_rn(a3, *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2))));
+                    }
+                    dst4[(size_t)gl * 32] = make_float4(__fmul_rn(a0, scale), __fmul_rn(a1, scale),
+                                                        __fmul_rn(a2, scale), __fmul_rn(a3, scale));
+                }
+            }
+        }
+
+        for (int64_t g = g_rest + warp; g < g_end; g += kWarps) {
             const int64_t i0 = (g << 7) + 4 * lane;
             if (i0 >= n) continue;
             const int64_t bit = i0 * BITS;
@@ -185,8 +291,7 @@ k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* _
                 const uint32_t bits4 = __funnelshift_r(w_lo, w_hi, sh) & kMask4;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    uint32_t code = (bits4 >> (j * BITS)) & kMask1;
-                    if (code > (uint32_t)(s - 1)) code = (uint32_t)(s - 1);
+                    const uint32_t code = (bits4 >> (j * BITS)) & kMask1;
                     acc[j] = __fadd_rn(acc[j], sh_lv[k][code]);
                 }
             }
@@ -215,11 +320,11 @@ cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int 
                                  uint32_t* d_packed, int sm_count, cudaStream_t stream)
 {
     FlatGrid g = make_flat_grid(total, flat_target(sm_count), 8192);
-    const uint32_t slo = (uint32_t)seed, shi = (uint32_t)(seed >> 32);
+    const PhiloxKeys keys = philox_round_keys((uint32_t)seed, (uint32_t)(seed >> 32));
     const int bits = ogq_bits_for_levels(s);
 #define OGQ_LAUNCH_Q(B, TH)                                                                          \
     k_quantize_pack<B, TH><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, s,     \
-                                                            d_levels, d_thresh, slo, shi, stream_id, \
+                                                            d_levels, d_thresh, keys, stream_id,     \
                                                             d_packed_off, d_packed)
     launch_begin(scheme == OGQ_BINGRAD_B ? "k_quantize_pack_threshold" : "k_quantize_pack_random", stream);
     if (scheme == OGQ_BINGRAD_B) {

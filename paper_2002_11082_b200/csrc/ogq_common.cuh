@@ -133,6 +133,37 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
+// The ten round keys of one Philox4x32-10 key (the Weyl sequence of the key schedule), computed on
+// the host and handed to a kernel by value: a kernel parameter can be an ALU operand directly, so the
+// schedule costs no instruction on the device.
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+};
+
+inline PhiloxKeys philox_round_keys(uint32_t k0, uint32_t k1)
+{
+    PhiloxKeys K;
+    for (int r = 0; r < 10; ++r) {
+        K.k0[r] = k0 + (uint32_t)r * 0x9E3779B9u;
+        K.k1[r] = k1 + (uint32_t)r * 0xBB67AE85u;
+    }
+    return K;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKeys& K)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c0 = n0; c1 = (uint32_t)p1; c2 = n2; c3 = (uint32_t)p0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
 // ---------------------------------------------------------------------------
 // Warp / block reductions with a fixed combination order (reproducible).
 // ---------------------------------------------------------------------------

@@ -145,6 +145,24 @@ __device__ __forceinline__ void table_from_intervals(Table& tb, const Interval* 
     tb.ncells = nc;
 }
 
+// The same, spread over the first kMaxIv threads of the CTA (called by all threads; the caller
+// synchronises afterwards).
+__device__ __forceinline__ void table_from_intervals_cta(Table& tb, const Interval* iv, int m)
+{
+    const int j = threadIdx.x;
+    if (j < kMaxIv) {
+        if (j < m) {
+            tb.klo[j] = iv[j].klo; tb.khi[j] = iv[j].khi; tb.sh[j] = iv[j].sh; tb.cellbase[j] = iv[j].cellbase;
+        } else {
+            tb.klo[j] = 0xffffffffu; tb.khi[j] = 0u; tb.sh[j] = 0; tb.cellbase[j] = 0;
+        }
+    }
+    if (j == 0) {
+        tb.m = m;
+        tb.ncells = (m > 0) ? iv[m - 1].cellbase + iv[m - 1].ncell : 0;
+    }
+}
+
 // Round-1 intervals: coarse (one cell per binade) outside a window of kSelW binades that ends
 // at binade hi_e, fine inside.  Negative values only for signed keys.
 __device__ __forceinline__ int round1_intervals(int hi_e, bool magnitude_only, Interval* iv)
@@ -331,37 +349,93 @@ __device__ __forceinline__ void visit_plain(const float* __restrict__ grad, int6
 // max are tracked as floats; -0 is folded into +0 by adding +0 first.
 constexpr int64_t kR1MaxPiece = (int64_t)1 << 16;
 
+__device__ __forceinline__ float min3f(float a, float b, float c)
+{
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));  // a NaN operand is skipped
+    return r;
+}
+__device__ __forceinline__ float max3f(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// shared-memory add without a return value, on a 32-bit shared address
+__device__ __forceinline__ void red_shared_add(uint32_t addr, uint32_t v)
+{
+    asm volatile("red.shared.add.u32 [%0], %1;" :: "r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t atom_shared_add(uint32_t addr, uint32_t v)
+{
+    uint32_t old;
+    asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+    return old;
+}
+
 template <bool MAG>
 struct Round1Body {
     uint32_t lo23;
     int lo_e;
-    uint32_t* cnt;  // counts, already offset to the first non-negative magnitude cell; low sums at
-                    // + kCells, their carries at + 2 kCells
+    uint32_t cnt;  // shared address of the count of the first non-negative magnitude cell; the low
+                   // sums lie kCells words above the counts, their carries 2 kCells words above
     float mn, mx;
     uint32_t nonfinite;
 
-    __device__ __forceinline__ void operator()(float v)
+    static __device__ __forceinline__ float canon(float v) { return (MAG ? fabsf(v) : v) + 0.0f; }
+
+    // a value inside the fine window (rel = magnitude bits - lo23 < kSelW << 23)
+    __device__ __forceinline__ void fine(uint32_t bits, uint32_t rel)
     {
-        v = (MAG ? fabsf(v) : v) + 0.0f;
-        const uint32_t bits = __float_as_uint(v);
         const int sgn = MAG ? 0 : ((int)bits >> 31);  // 0 or -1
-        const uint32_t mag = MAG ? bits : (bits & 0x7fffffffu);
+        const uint32_t c = cnt + (uint32_t)(((lo_e + (int)(rel >> (23 - kSelM))) ^ sgn) << 2);
+        red_shared_add(c, 1u);
+        red_shared_add(c + 4u * kCells, (bits ^ (uint32_t)sgn) & ((1u << (23 - kSelM)) - 1u));
+    }
+
+    // any value (already canonical)
+    __device__ __forceinline__ void any(uint32_t bits)
+    {
+        const int sgn = MAG ? 0 : ((int)bits >> 31);
+        const uint32_t mag = bits & 0x7fffffffu;
         const uint32_t rel = mag - lo23;
-        mn = fminf(mn, v);
-        mx = fmaxf(mx, v);
         if (rel < ((uint32_t)kSelW << 23)) {
-            uint32_t* c = cnt + ((lo_e + (int)(rel >> (23 - kSelM))) ^ sgn);
-            atomicAdd(c, 1u);
-            atomicAdd(c + kCells, (mag ^ (uint32_t)sgn) & ((1u << (23 - kSelM)) - 1u));
+            fine(bits, rel);
         } else {  // outside the fine window: one cell per binade
             const int e = (int)(mag >> 23);
             const int mi = (e < lo_e) ? e : e - kSelW + (kSelW << kSelM);
             if (e == 255) nonfinite = 1u;  // the window never reaches binade 255
-            uint32_t* c = cnt + (mi ^ sgn);
+            const uint32_t c = cnt + (uint32_t)((mi ^ sgn) << 2);
             const uint32_t low = (mag ^ (uint32_t)sgn) & 0x7fffffu;
-            atomicAdd(c, 1u);
-            const uint32_t old = atomicAdd(c + kCells, low);
-            if (old + low < old) atomicAdd(c + 2 * kCells, 1u);
+            red_shared_add(c, 1u);
+            const uint32_t old = atom_shared_add(c + 4u * kCells, low);
+            if (old + low < old) red_shared_add(c + 8u * kCells, 1u);
+        }
+    }
+
+    __device__ __forceinline__ void one(float v)
+    {
+        v = canon(v);
+        mn = fminf(mn, v);
+        mx = fmaxf(mx, v);
+        any(__float_as_uint(v));
+    }
+
+    __device__ __forceinline__ void four(float4 x)
+    {
+        const float v0 = canon(x.x), v1 = canon(x.y), v2 = canon(x.z), v3 = canon(x.w);
+        mn = min3f(min3f(mn, v0, v1), v2, v3);
+        mx = max3f(max3f(mx, v0, v1), v2, v3);
+        const uint32_t b0 = __float_as_uint(v0), b1 = __float_as_uint(v1), b2 = __float_as_uint(v2),
+                       b3 = __float_as_uint(v3);
+        const uint32_t r0 = (b0 & 0x7fffffffu) - lo23, r1 = (b1 & 0x7fffffffu) - lo23,
+                       r2 = (b2 & 0x7fffffffu) - lo23, r3 = (b3 & 0x7fffffffu) - lo23;
+        // the window spans kSelW = 2^4 binades, so "all four inside" is one test on the OR
+        static_assert((kSelW & (kSelW - 1)) == 0, "window size must be a power of two");
+        if ((r0 | r1 | r2 | r3) < ((uint32_t)kSelW << 23)) {
+            fine(b0, r0); fine(b1, r1); fine(b2, r2); fine(b3, r3);
+        } else {
+            any(b0); any(b1); any(b2); any(b3);
         }
     }
 };
@@ -373,15 +447,15 @@ __device__ __forceinline__ void stream_round1(const float* __restrict__ grad, in
     Round1Body<MAG> f;
     f.lo23 = (uint32_t)lo_e << 23;
     f.lo_e = lo_e;
-    f.cnt = hist + (MAG ? 0 : kRound1Mag);
+    f.cnt = (uint32_t)__cvta_generic_to_shared(hist + (MAG ? 0 : kRound1Mag));
     f.mn = vmin; f.mx = vmax; f.nonfinite = nonfinite;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
     int64_t b = pe & ~(int64_t)3;
     if (b < a) b = a;
     const int tid = threadIdx.x;
-    if (tid < (int)(a - pb)) f(__ldg(grad + pb + tid));
-    if (tid < (int)(pe - b)) f(__ldg(grad + b + tid));
+    if (tid < (int)(a - pb)) f.one(__ldg(grad + pb + tid));
+    if (tid < (int)(pe - b)) f.one(__ldg(grad + b + tid));
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     int64_t i = (a >> 2) + tid;
     const int64_t e = b >> 2;
@@ -390,12 +464,9 @@ __device__ __forceinline__ void stream_round1(const float* __restrict__ grad, in
 #pragma unroll
         for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i + u * kSelThreads);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { f(x[u].x); f(x[u].y); f(x[u].z); f(x[u].w); }
+        for (int u = 0; u < 4; ++u) f.four(x[u]);
     }
-    for (; i < e; i += kSelThreads) {
-        const float4 x = __ldg(g4 + i);
-        f(x.x); f(x.y); f(x.z); f(x.w);
-    }
+    for (; i < e; i += kSelThreads) f.four(__ldg(g4 + i));
     vmin = f.mn; vmax = f.mx; nonfinite = f.nonfinite;
 }
 
@@ -466,17 +537,20 @@ __device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
 }
 
 struct Round2Warp {
-    const uint32_t* coarse;  // the table's prefilter bitmap
-    uint32_t* stage;         // this warp's kStageCap parking slots
-    int* fillp;              // their fill counter (shared memory, bumped by the lanes that hit)
+    uint32_t coarse;  // shared addresses: the table's prefilter bitmap,
+    uint32_t stage;   // this warp's kStageCap parking slots,
+    uint32_t fillp;   // and their fill counter (bumped by the lanes that hit)
 
     // Phase A for one element: no warp collective, only the lanes that pass the bitmap test do work.
     __device__ __forceinline__ void one(float v)
     {
         const uint32_t bits = __float_as_uint(v);
-        const uint32_t word = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(coarse) +
-                                                                 ((bits >> 20) & 0xffcu));
-        if (__funnelshift_r(word, 0u, bits >> 17) & 1u) stage[atomicAdd(fillp, 1)] = bits;
+        uint32_t word;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(coarse + ((bits >> 20) & 0xffcu)));
+        if (__funnelshift_r(word, 0u, bits >> 17) & 1u) {
+            const uint32_t pos = atom_shared_add(fillp, 1u);
+            asm volatile("st.shared.u32 [%0], %1;" :: "r"(stage + (pos << 2)), "r"(bits) : "memory");
+        }
     }
 };
 
@@ -496,7 +570,9 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
     if (lane == 0) fills[warp] = 0;
     __syncthreads();
     Round2Warp w;
-    w.coarse = tb.coarse; w.stage = stage; w.fillp = &fills[warp];
+    w.coarse = (uint32_t)__cvta_generic_to_shared(tb.coarse);
+    w.stage = (uint32_t)__cvta_generic_to_shared(stage);
+    w.fillp = (uint32_t)__cvta_generic_to_shared(&fills[warp]);
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
     int64_t b = pe & ~(int64_t)3;
@@ -509,10 +585,10 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
     // at most 32 * 16 = 512 values are parked between two checks, and the stage holds kStageCap = 1024
     auto check = [&]() {
         __syncwarp();
-        const int f = *(volatile int*)w.fillp;
+        const int f = *(volatile int*)&fills[warp];
         if (f > kStageCap - 512) {
-            round2_drain(&tb, &ctx, w.stage, f);
-            if (lane == 0) *w.fillp = 0;
+            round2_drain(&tb, &ctx, stage, f);
+            if (lane == 0) fills[warp] = 0;
             __syncwarp();
         }
     };
@@ -539,7 +615,7 @@ __device__ __forceinline__ void stream_round2(const float* __restrict__ grad, in
         check();
     }
     __syncwarp();
-    round2_drain(&tb, &ctx, w.stage, *(volatile int*)w.fillp);
+    round2_drain(&tb, &ctx, stage, *(volatile int*)&fills[warp]);
 }
 
 // Streams one piece of a tensor's working set: histogram of the keys inside the intervals,
@@ -1626,27 +1702,28 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round2(SelArgs A)
         TState* st = A.ws.st + t;
         if (__ldcg(&st->done)) return;
         __syncthreads();
-        if (threadIdx.x == 0) {
-            table_from_intervals(tb, st->iv, __ldcg(&st->m));
-            tb.lo_e = st->hi_e - kSelW;
-        }
+        table_from_intervals_cta(tb, st->iv, __ldcg(&st->m));
         __syncthreads();
         build_prefilter(tb, pb);
         zero_hist(hist, tb.ncells);
         __syncthreads();
+        OGQ_CTA_PHASE(0);
         stream_round2(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells,
                       reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
                       A.ws.buf[0] + tbeg, &st->cursor[0]);
         __syncthreads();
+        OGQ_CTA_PHASE(1);
         flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         __threadfence();
         __syncthreads();
+        OGQ_CTA_PHASE(2);
         const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
         if (threadIdx.x == 0) {
             const unsigned prev = atomicAdd(&st->arrive, 1u);
             sh_last = (prev == (unsigned)(c1 - c0));
         }
         __syncthreads();
+        OGQ_CTA_PHASE(3);
         if (!sh_last) return;
         __threadfence();
         OGQ_CTA_SOLVER(solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme,

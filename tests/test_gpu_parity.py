@@ -233,7 +233,7 @@ def test_quantize_special_values_and_duplicate_levels():
 # ------------------------------------------------------------------ unpack + sum
 
 
-@pytest.mark.parametrize("s,K", [(2, 1), (3, 4), (5, 3), (9, 8), (17, 2)])
+@pytest.mark.parametrize("s,K", [(2, 1), (3, 4), (5, 3), (9, 8), (17, 2), (9, 11), (9, 17), (3, 9), (2, 3)])
 @pytest.mark.parametrize("bucket_fn", [wl.config2, ragged_bucket])
 def test_unpack_sum(bucket_fn, s, K):
     base = bucket_fn()
