@@ -32,6 +32,7 @@ constexpr int kSelW = 16;          // binades in the fine window of round 1
 constexpr int kSelM = 7;           // log2(cells per binade) in the window
 constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
 constexpr int kMidN = 131072;      // tensors up to this size are solved start to finish by one CTA of their own
+constexpr int64_t kSelMinChunk = 196608;  // elements per flat streaming CTA, at least
 constexpr int kStageCap = 1024;    // per-warp staging entries for compaction
 constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
 constexpr int kSliceElems = 16384;
@@ -1815,7 +1816,13 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
         e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
     }
-    int target = sm_count * 4 < kMaxFlatCtas ? sm_count * 4 : kMaxFlatCtas;
+    // Flat streaming CTAs (one is resident per SM): each pays a set-up, a flush of its cells and an
+    // arrival, so they get at least kSelMinChunk elements; between one and two CTAs per SM, the more
+    // the better the balance against the per-tensor CTAs of the same grid.
+    int64_t want = total / kSelMinChunk;
+    if (want < sm_count) want = sm_count;
+    if (want > 2 * (int64_t)sm_count) want = 2 * (int64_t)sm_count;
+    const int target = want < kMaxFlatCtas ? (int)want : kMaxFlatCtas;
     FlatGrid g = make_flat_grid(total, target, 65536);
     SelArgs A;
     A.grad = d_grad; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
