@@ -442,7 +442,7 @@ struct Round1Body {
 };
 
 template <bool MAG>
-__device__ __forceinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe, int lo_e,
+__device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe, int lo_e,
                                               uint32_t* hist, float& vmin, float& vmax, uint32_t& nonfinite)
 {
     Round1Body<MAG> f;
@@ -555,7 +555,7 @@ struct Round2Warp {
     }
 };
 
-__device__ __forceinline__ void stream_round2(const float* __restrict__ grad, int64_t pb, int64_t pe,
+__device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64_t pb, int64_t pe,
                                               bool magnitude_only, const Table& tb, uint32_t* cnt, uint32_t* lo,
                                               uint32_t* hi, uint32_t* stage, uint32_t* dst,
                                               unsigned long long* cursor)
