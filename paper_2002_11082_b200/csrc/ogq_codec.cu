@@ -17,34 +17,17 @@ namespace ogq {
 constexpr int kMaxLevels = 32;
 constexpr int kMaxWorkers = 64;
 
-// OR-combine the 4*BITS-bit chunk of each lane into words.  For BITS = 1, 2, 4 a word is made of
-// 8, 4, 2 neighbouring lanes and the first lane of each such set returns it (word index lane / L);
-// for BITS = 3, 5 eight lanes make BITS words and lane (8q + j), j < BITS, returns word j of set q.
+// OR-combine the 4*BITS-bit chunk of each lane into words, BITS = 1, 2 or 4: a word is made of
+// 8, 4, 2 neighbouring lanes and the first lane of each such set returns it (word index lane / L).
 template <int BITS>
 __device__ __forceinline__ uint32_t assemble_words(uint32_t chunk, int lane)
 {
-    if (BITS == 1 || BITS == 2 || BITS == 4) {
-        constexpr int L = 8 / BITS;
-        uint32_t x = chunk << (4 * BITS * (lane & (L - 1)));
+    static_assert(BITS == 1 || BITS == 2 || BITS == 4, "other widths are combined in shared memory");
+    constexpr int L = 8 / BITS;
+    uint32_t x = chunk << (4 * BITS * (lane & (L - 1)));
 #pragma unroll
-        for (int o = 1; o < L; o <<= 1) x |= __shfl_xor_sync(0xffffffffu, x, o);
-        return x;
-    }
-    const int j = lane & 7;
-    const int bitpos = j * 4 * BITS;
-    const int w0 = bitpos >> 5, sh = bitpos & 31;
-    const uint32_t lo = chunk << sh;
-    const uint32_t hi = (sh + 4 * BITS > 32) ? (chunk >> (32 - sh)) : 0u;
-    uint32_t mine = 0;
-#pragma unroll
-    for (int k = 0; k < BITS; ++k) {
-        uint32_t val = ((w0 == k) ? lo : 0u) | ((w0 + 1 == k) ? hi : 0u);
-        val |= __shfl_xor_sync(0xffffffffu, val, 1);
-        val |= __shfl_xor_sync(0xffffffffu, val, 2);
-        val |= __shfl_xor_sync(0xffffffffu, val, 4);
-        if (j == k) mine = val;
-    }
-    return mine;
+    for (int o = 1; o < L; o <<= 1) x |= __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
 }
 
 template <int BITS, bool THRESHOLD>
@@ -57,6 +40,10 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
     __shared__ float sh_lv[kMaxLevels];
     __shared__ float sh_w[kMaxLevels];
     __shared__ float2 sh_tab[kMaxLevels];  // {level k, width of the segment above it}
+    // 3- and 5-bit codes: the 4*BITS words of a warp's group are OR-ed together here (kept zero between uses)
+    __shared__ uint32_t sh_words[kWarps][(BITS == 3 || BITS == 5) ? 4 * BITS : 1];
+    if ((BITS == 3 || BITS == 5) && (threadIdx.x & 31) < 4 * BITS) sh_words[threadIdx.x >> 5][threadIdx.x & 31] = 0u;
+    __syncthreads();
 
     const int64_t lo = (int64_t)blockIdx.x * chunk;
     const int64_t hi = (lo + chunk < total) ? lo + chunk : total;
@@ -90,17 +77,27 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
         // per warp, no bounds checks.  The generic loop below takes what is left (the last, partial
         // group; everything when the tensor does not start on a 16-byte boundary).
         int64_t g_rest = g_beg;
-        if (!THRESHOLD && (BITS == 1 || BITS == 2 || BITS == 4) && aligned) {
+        if (aligned) {
             const int64_t g_full = (n >> 7) < g_end ? (n >> 7) : g_end;
             if (g_full > g_beg) {
                 g_rest = g_full;
-                constexpr int L = 8 / BITS;
+                constexpr bool kPow2 = (BITS == 1 || BITS == 2 || BITS == 4);
+                constexpr int L = kPow2 ? 8 / BITS : 1;  // lanes per word when a word is a whole number of lanes
                 const int ng = (int)(g_full - g_beg);
                 const float4* src = reinterpret_cast<const float4*>(base + (g_beg << 7)) + lane;
-                uint32_t* dstw = out + g_beg * (4 * BITS) + lane / L;
+                // which word of the group this lane stores: the first lane of each set of L lanes (see
+                // assemble_words), or, for 3 and 5 bits, lane w stores word w after the shared-memory OR
+                const bool writer = kPow2 ? (lane & (L - 1)) == 0 : lane < 4 * BITS;
+                uint32_t* dstw = out + g_beg * (4 * BITS) + (kPow2 ? lane / L : lane);
+                uint32_t* wsm = sh_words[warp];
+                const int obit = (lane * 4 * BITS) & 31, oword = (lane * 4 * BITS) >> 5;  // kPow2 == false only
                 const uint64_t q0 = ((uint64_t)g_beg << 5) + (uint64_t)lane;
-                const bool writer = (lane & (L - 1)) == 0;
                 auto code4 = [&](const float4 v, int gl) -> uint32_t {
+                    if constexpr (THRESHOLD) {
+                        const uint32_t b4 = ((v.x >= b0) ? 1u : 0u) | ((v.y >= b0) ? 2u : 0u) |
+                                            ((v.z >= b0) ? 4u : 0u) | ((v.w >= b0) ? 8u : 0u);
+                        return assemble_words<BITS>(b4, lane);
+                    }
                     const uint64_t q = q0 + ((uint64_t)(uint32_t)gl << 5);
                     const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)t, stream_id, keys);
                     const float xs[4] = {v.x, v.y, v.z, v.w};
@@ -117,7 +114,17 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                         const float rhs = __fmul_rn(__fsub_rn(xs[j], e.x), 16777216.0f);
                         bits4 |= ((uint32_t)idx + ((lhs < rhs) ? 1u : 0u)) << (j * BITS);
                     }
-                    return assemble_words<BITS>(bits4, lane);
+                    if constexpr (kPow2) {
+                        return assemble_words<BITS>(bits4, lane);
+                    } else {
+                        // a lane's 4*BITS bits touch at most two words of the group
+                        atomicOr(wsm + oword, bits4 << obit);
+                        if (obit + 4 * BITS > 32) atomicOr(wsm + oword + 1, bits4 >> (32 - obit));
+                        __syncwarp();
+                        const uint32_t word = writer ? atomicExch(wsm + lane, 0u) : 0u;
+                        __syncwarp();
+                        return word;
+                    }
                 };
                 // software pipeline: the loads of the next two groups are issued before the current two
                 // are quantized
@@ -177,19 +184,26 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                     if (i0 + j >= n) c[j] = 0u;  // zero padding beyond the tensor
             }
             const uint32_t bits4 = c[0] | (c[1] << BITS) | (c[2] << (2 * BITS)) | (c[3] << (3 * BITS));
-            const uint32_t word = assemble_words<BITS>(bits4, lane);
-            if (BITS == 1 || BITS == 2 || BITS == 4) {
+            if constexpr (BITS == 1 || BITS == 2 || BITS == 4) {
+                const uint32_t word = assemble_words<BITS>(bits4, lane);
                 constexpr int L = 8 / (BITS == 3 || BITS == 5 ? 1 : BITS);
                 if ((lane & (L - 1)) == 0) {
                     const int64_t widx = g * (4 * BITS) + lane / L;
                     if (widx < region) out[widx] = word;
                 }
             } else {
-                const int j8 = lane & 7;
-                if (j8 < BITS) {
-                    const int64_t widx = g * (4 * BITS) + (lane >> 3) * BITS + j8;
+                // 3 and 5 bits: OR the lanes' bits into the group's 4*BITS words in shared memory
+                uint32_t* wsm = sh_words[warp];
+                const int obit = (lane * 4 * BITS) & 31, oword = (lane * 4 * BITS) >> 5;
+                atomicOr(wsm + oword, bits4 << obit);
+                if (obit + 4 * BITS > 32) atomicOr(wsm + oword + 1, bits4 >> (32 - obit));
+                __syncwarp();
+                if (lane < 4 * BITS) {
+                    const uint32_t word = atomicExch(wsm + lane, 0u);
+                    const int64_t widx = g * (4 * BITS) + lane;
                     if (widx < region) out[widx] = word;
                 }
+                __syncwarp();
             }
         }
     });
