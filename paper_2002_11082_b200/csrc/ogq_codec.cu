@@ -30,6 +30,36 @@ __device__ __forceinline__ uint32_t assemble_words(uint32_t chunk, int lane)
     return x;
 }
 
+// Segment search and rounding decision of one element on the fast path.  `tabaddr` is the shared
+// address of the table {level k, width of the segment above it} (8 bytes per entry) and `mid` its
+// middle level.  Returns the address of the entry whose index is the element's code: the entry of the
+// segment's lower level, or the next one when the element rounds up.  The halving steps are written
+// as "load, compare, predicated add" so that each costs three instructions.
+template <int STEP>
+__device__ __forceinline__ void search_step(uint32_t& a, float v)
+{
+    asm("{ .reg .pred p; .reg .f32 t; ld.shared.f32 t, [%0+%2]; setp.le.f32 p, t, %1; @p add.u32 %0, %0, %2; }"
+        : "+r"(a) : "f"(v), "n"(STEP * 8));
+}
+
+template <int BITS>
+__device__ __forceinline__ uint32_t entry_after_rounding(float v, uint32_t rnd, uint32_t tabaddr, float mid)
+{
+    uint32_t a = tabaddr;
+    if constexpr (BITS >= 2) {
+        if (mid <= v) a += 8u << (BITS - 2);
+        if constexpr (BITS >= 5) search_step<4>(a, v);
+        if constexpr (BITS >= 4) search_step<2>(a, v);
+        if constexpr (BITS >= 3) search_step<1>(a, v);
+    }
+    float lo, w;
+    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(lo), "=f"(w) : "r"(a));
+    const float lhs = __fmul_rn((float)(rnd >> 8), w);
+    const float rhs = __fmul_rn(__fsub_rn(v, lo), 16777216.0f);
+    asm("{ .reg .pred p; setp.lt.f32 p, %1, %2; @p add.u32 %0, %0, 8; }" : "+r"(a) : "f"(lhs), "f"(rhs));
+    return a;
+}
+
 template <int BITS, bool THRESHOLD>
 __global__ void __launch_bounds__(kThreads)
 k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off, int T, int64_t total,
@@ -73,11 +103,12 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
         const bool aligned = (tb & 3) == 0;
         const float* base = grad + tb;
 
-        // Fast path: groups that lie wholly inside the tensor, 128-bit loads, two groups in flight
+        // Fast path: groups that lie wholly inside the tensor, 128-bit loads, four groups in flight
         // per warp, no bounds checks.  The generic loop below takes what is left (the last, partial
-        // group; everything when the tensor does not start on a 16-byte boundary).
+        // group; everything when the tensor does not start on a 16-byte boundary, or when its Philox
+        // counters do not fit 32 bits).
         int64_t g_rest = g_beg;
-        if (aligned) {
+        if (aligned && n <= ((int64_t)1 << 34)) {
             const int64_t g_full = (n >> 7) < g_end ? (n >> 7) : g_end;
             if (g_full > g_beg) {
                 g_rest = g_full;
@@ -91,58 +122,55 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                 uint32_t* dstw = out + g_beg * (4 * BITS) + (kPow2 ? lane / L : lane);
                 uint32_t* wsm = sh_words[warp];
                 const int obit = (lane * 4 * BITS) & 31, oword = (lane * 4 * BITS) >> 5;  // kPow2 == false only
-                const uint64_t q0 = ((uint64_t)g_beg << 5) + (uint64_t)lane;
+                const uint32_t c0_first = (uint32_t)(g_beg << 5) + (uint32_t)lane;  // counters fit 32 bits here
+                const uint32_t tabaddr = (uint32_t)__cvta_generic_to_shared(sh_tab);
+                // the sum of the four entry addresses of a lane carries this multiple of the table's base
+                const uint32_t tab4 = tabaddr * (1u + (1u << BITS) + (1u << (2 * BITS)) + (1u << (3 * BITS)));
+                float mid = 0.f;
+                PhiloxHoist hz = {};
+                if constexpr (!THRESHOLD) {
+                    mid = sh_tab[(BITS >= 2) ? (1 << (BITS - 2)) : 0].x;
+                    hz = philox_hoist(0u, (uint32_t)t, stream_id, keys);
+                }
                 auto code4 = [&](const float4 v, int gl) -> uint32_t {
                     if constexpr (THRESHOLD) {
                         const uint32_t b4 = ((v.x >= b0) ? 1u : 0u) | ((v.y >= b0) ? 2u : 0u) |
                                             ((v.z >= b0) ? 4u : 0u) | ((v.w >= b0) ? 8u : 0u);
                         return assemble_words<BITS>(b4, lane);
-                    }
-                    const uint64_t q = q0 + ((uint64_t)(uint32_t)gl << 5);
-                    const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)t, stream_id, keys);
-                    const float xs[4] = {v.x, v.y, v.z, v.w};
-                    const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-                    uint32_t bits4 = 0u;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        int idx = 0;
-#pragma unroll
-                        for (int step = (BITS >= 2) ? (1 << (BITS - 2)) : 0; step >= 1; step >>= 1)
-                            if (sh_tab[idx + step].x <= xs[j]) idx += step;
-                        const float2 e = sh_tab[idx];
-                        const float lhs = __fmul_rn((float)(rw[j] >> 8), e.y);
-                        const float rhs = __fmul_rn(__fsub_rn(xs[j], e.x), 16777216.0f);
-                        bits4 |= ((uint32_t)idx + ((lhs < rhs) ? 1u : 0u)) << (j * BITS);
-                    }
-                    if constexpr (kPow2) {
-                        return assemble_words<BITS>(bits4, lane);
                     } else {
-                        // a lane's 4*BITS bits touch at most two words of the group
-                        atomicOr(wsm + oword, bits4 << obit);
-                        if (obit + 4 * BITS > 32) atomicOr(wsm + oword + 1, bits4 >> (32 - obit));
-                        __syncwarp();
-                        const uint32_t word = writer ? atomicExch(wsm + lane, 0u) : 0u;
-                        __syncwarp();
-                        return word;
+                        const uint4 r = philox4x32_10_tail(c0_first + ((uint32_t)gl << 5), hz, keys);
+                        const uint32_t a0 = entry_after_rounding<BITS>(v.x, r.x, tabaddr, mid),
+                                       a1 = entry_after_rounding<BITS>(v.y, r.y, tabaddr, mid),
+                                       a2 = entry_after_rounding<BITS>(v.z, r.z, tabaddr, mid),
+                                       a3 = entry_after_rounding<BITS>(v.w, r.w, tabaddr, mid);
+                        // entries are 8 bytes apart: (address - base) / 8 is the code
+                        const uint32_t bits4 =
+                            (a0 + (a1 << BITS) + (a2 << (2 * BITS)) + (a3 << (3 * BITS)) - tab4) >> 3;
+                        if constexpr (kPow2) {
+                            return assemble_words<BITS>(bits4, lane);
+                        } else {
+                            // a lane's 4*BITS bits touch at most two words of the group
+                            atomicOr(wsm + oword, bits4 << obit);
+                            if (obit + 4 * BITS > 32) atomicOr(wsm + oword + 1, bits4 >> (32 - obit));
+                            __syncwarp();
+                            const uint32_t word = writer ? atomicExch(wsm + lane, 0u) : 0u;
+                            __syncwarp();
+                            return word;
+                        }
                     }
                 };
-                // software pipeline: the loads of the next two groups are issued before the current two
-                // are quantized
-                int gl = warp;
-                const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                float4 va = (gl < ng) ? __ldg(src + (size_t)gl * 32) : zero4;
-                float4 vb = (gl + kWarps < ng) ? __ldg(src + (size_t)(gl + kWarps) * 32) : zero4;
-                for (; gl < ng; gl += 2 * kWarps) {
-                    const int gn = gl + 2 * kWarps;
-                    const float4 na = (gn < ng) ? __ldg(src + (size_t)gn * 32) : zero4;
-                    const float4 nb = (gn + kWarps < ng) ? __ldg(src + (size_t)(gn + kWarps) * 32) : zero4;
-                    const uint32_t wa = code4(va, gl);
-                    if (writer) dstw[(size_t)gl * (4 * BITS)] = wa;
-                    if (gl + kWarps < ng) {
-                        const uint32_t wb = code4(vb, gl + kWarps);
-                        if (writer) dstw[(size_t)(gl + kWarps) * (4 * BITS)] = wb;
-                    }
-                    va = na; vb = nb;
+                constexpr int U = 4;  // groups per warp and trip: all loads are issued before the first use
+                for (int gl = warp; gl < ng; gl += U * kWarps) {
+                    float4 v[U];
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+                        if (gl + u * kWarps < ng) v[u] = __ldg(src + (size_t)(gl + u * kWarps) * 32);
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+                        if (gl + u * kWarps < ng) {
+                            const uint32_t w = code4(v[u], gl + u * kWarps);
+                            if (writer) dstw[(size_t)(gl + u * kWarps) * (4 * BITS)] = w;
+                        }
                 }
             }
         }

@@ -164,6 +164,53 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
+// Rounds 1 and 2 of Philox4x32-10 split into the part that depends only on (c1, c2, c3) and the key,
+// computed once per tensor, and the part that depends on c0.  c1..c3 = (counter high word, tensor
+// index, stream id) are the same for every element of a tensor whose counters fit 32 bits: the
+// product of round 1's second multiplier, round 1's first output word and therefore round 2's first
+// product are all uniform.
+struct PhiloxHoist {
+    uint32_t n0;          // first word after round 1
+    uint32_t lo1;         // low half of round 1's second product (second word after round 1)
+    uint32_t c3k1;        // c3 ^ k1[0]
+    uint32_t hi0b, lo0b;  // round 2's first product (multiplier * n0)
+};
+
+__device__ __forceinline__ PhiloxHoist philox_hoist(uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys& K)
+{
+    PhiloxHoist h;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    h.n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[0];
+    h.lo1 = (uint32_t)p1;
+    h.c3k1 = c3 ^ K.k1[0];
+    const uint64_t p0b = (uint64_t)0xD2511F53u * h.n0;
+    h.hi0b = (uint32_t)(p0b >> 32);
+    h.lo0b = (uint32_t)p0b;
+    return h;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10_tail(uint32_t c0, const PhiloxHoist& h, const PhiloxKeys& K)
+{
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;  // round 1: only this product depends on c0
+    uint32_t a0, a1, a2 = (uint32_t)(p0 >> 32) ^ h.c3k1, a3 = (uint32_t)p0;
+    {  // round 2: the first product is uniform
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * a2;
+        a0 = (uint32_t)(p1 >> 32) ^ h.lo1 ^ K.k0[1];
+        a1 = (uint32_t)p1;
+        a2 = h.hi0b ^ a3 ^ K.k1[1];
+        a3 = h.lo0b;
+    }
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
+        const uint64_t q0 = (uint64_t)0xD2511F53u * a0;
+        const uint64_t q1 = (uint64_t)0xCD9E8D57u * a2;
+        const uint32_t n0 = (uint32_t)(q1 >> 32) ^ a1 ^ K.k0[r];
+        const uint32_t n2 = (uint32_t)(q0 >> 32) ^ a3 ^ K.k1[r];
+        a0 = n0; a1 = (uint32_t)q1; a2 = n2; a3 = (uint32_t)q0;
+    }
+    return make_uint4(a0, a1, a2, a3);
+}
+
 // ---------------------------------------------------------------------------
 // Warp / block reductions with a fixed combination order (reproducible).
 // ---------------------------------------------------------------------------
