@@ -26,14 +26,17 @@
 
 namespace ogq {
 
-constexpr int kSelThreads = 1024;   // one CTA per SM; 32 warps keep enough loads in flight
+constexpr int kSelThreads = 512;    // two CTAs are resident per SM: a CTA in a solver pass, a sort or a
+                                    // set-up phase leaves the other half of the SM streaming
+constexpr int kSelResident = 2;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelW = 16;          // binades in the fine window of round 1
 constexpr int kSelM = 7;           // log2(cells per binade) in the window
 constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
 constexpr int kMidN = 131072;      // tensors up to this size are solved start to finish by one CTA of their own
-constexpr int64_t kSelMinChunk = 196608;  // elements per flat streaming CTA, at least
-constexpr int kStageCap = 1024;    // per-warp staging entries for compaction
+constexpr int64_t kSelMinChunk = 98304;   // elements per flat streaming CTA, at least
+constexpr int kStageCap = 320;     // per-warp staging entries for compaction
+constexpr int kParkMax = 256;      // values one warp can park between two checks of round 2 (32 lanes x 8)
 constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
 constexpr int kSliceElems = 16384;
 constexpr int kMaxRounds = 32;
@@ -583,11 +586,11 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
         else if (lane >= 4 && lane - 4 < (int)(pe - b)) w.one(__ldg(grad + b + lane - 4));
         __syncwarp();
     }
-    // at most 32 * 16 = 512 values are parked between two checks, and the stage holds kStageCap = 1024
+    // at most kParkMax values are parked between two checks
     auto check = [&]() {
         __syncwarp();
         const int f = *(volatile int*)&fills[warp];
-        if (f > kStageCap - 512) {
+        if (f > kStageCap - kParkMax) {
             round2_drain(&tb, &ctx, stage, f);
             if (lane == 0) fills[warp] = 0;
             __syncwarp();
@@ -601,8 +604,10 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
 #pragma unroll
         for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i0 + lane + u * kSelThreads);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { w.one(x[u].x); w.one(x[u].y); w.one(x[u].z); w.one(x[u].w); }
-        check();
+        for (int u = 0; u < 4; ++u) {
+            w.one(x[u].x); w.one(x[u].y); w.one(x[u].z); w.one(x[u].w);
+            if (u & 1) check();
+        }
     }
     if (i0 < e) {
 #pragma unroll
@@ -612,8 +617,8 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
                 const float4 x = __ldg(g4 + i);
                 w.one(x.x); w.one(x.y); w.one(x.z); w.one(x.w);
             }
+            if (u & 1) check();
         }
-        check();
     }
     __syncwarp();
     round2_drain(&tb, &ctx, stage, *(volatile int*)&fills[warp]);
@@ -1507,7 +1512,7 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
     }
 }
 
-__global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
+__global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ Table tb;
@@ -1537,7 +1542,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
             __syncthreads();  // earlier readers of sh_i are done
             if ((threadIdx.x & 31) == 0) sh_i[threadIdx.x >> 5] = e;
             __syncthreads();
-            hi_e = __reduce_max_sync(0xffffffffu, sh_i[threadIdx.x & 31]) + 2;
+            hi_e = __reduce_max_sync(0xffffffffu, ((threadIdx.x & 31) < kSelWarps) ? sh_i[threadIdx.x & 31] : 0) + 2;
             if (hi_e < kSelW) hi_e = kSelW;
             if (hi_e > 255) hi_e = 255;  // binade 255 (Inf / NaN) always stays outside the fine window
         }
@@ -1640,6 +1645,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
     if ((int)blockIdx.x < A.T) {
         // the first T CTAs, one per tensor, settle the empty, small and mid-size tensors; they come
         // first in the grid because the mid-size ones run longest
+        [&]() {
         const int t = blockIdx.x;
         const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
         const int64_t n = tend - tbeg;
@@ -1673,6 +1679,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
                 return;
             finish_alone(A, t, smem, tb, S);
         }
+        }();
+        OGQ_CTA_END();
         return;
     }
 
@@ -1685,7 +1693,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round1(SelArgs A)
     OGQ_CTA_END();
 }
 
-__global__ void __launch_bounds__(kSelThreads, 1) k_sel_round2(SelArgs A)
+__global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ Table tb;
@@ -1733,7 +1741,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_sel_round2(SelArgs A)
     OGQ_CTA_END();
 }
 
-__global__ void __launch_bounds__(kSelThreads, 1) k_sel_round3(SelArgs A)
+__global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ Table tb;
@@ -1816,14 +1824,15 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
         e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
     }
-    // Flat streaming CTAs (one is resident per SM): each pays a set-up, a flush of its cells and an
-    // arrival, so they get at least kSelMinChunk elements; between one and two CTAs per SM, the more
+    // Flat streaming CTAs (kSelResident are resident per SM): each pays a set-up, a flush of its cells
+    // and an arrival, so they get at least kSelMinChunk elements; between one and two waves, the more
     // the better the balance against the per-tensor CTAs of the same grid.
+    const int64_t wave = (int64_t)kSelResident * sm_count;
     int64_t want = total / kSelMinChunk;
-    if (want < sm_count) want = sm_count;
-    if (want > 2 * (int64_t)sm_count) want = 2 * (int64_t)sm_count;
+    if (want < wave) want = wave;
+    if (want > 2 * wave) want = 2 * wave;
     const int target = want < kMaxFlatCtas ? (int)want : kMaxFlatCtas;
-    FlatGrid g = make_flat_grid(total, target, 65536);
+    FlatGrid g = make_flat_grid(total, target, 32768);
     SelArgs A;
     A.grad = d_grad; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
     A.scheme = scheme; A.s = s; A.levels = d_levels; A.status = d_status;
@@ -1837,7 +1846,7 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     k_sel_round2<<<g.ctas, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     launch_begin("k_sel_round3", stream);
-    k_sel_round3<<<sm_count, kSelThreads, kSmemBytes, stream>>>(A);
+    k_sel_round3<<<kSelResident * sm_count, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     return cudaGetLastError();
 }
