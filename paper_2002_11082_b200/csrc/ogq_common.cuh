@@ -36,13 +36,21 @@ inline FlatGrid make_flat_grid(int64_t total, int target_ctas, int64_t min_chunk
     return g;
 }
 
-// Largest t < T with off[t] <= x (the tensor that contains flat index x).
+// Largest t < T with off[t] <= x (the tensor that contains flat index x; 0 when there is none).
+// Called by all 32 lanes of a warp with the same arguments: every step probes 32 evenly spaced
+// offsets at once, so a bucket of a few hundred tensors costs two dependent loads instead of eight.
 __device__ __forceinline__ int find_tensor(const int64_t* __restrict__ off, int T, int64_t x)
 {
+    const int lane = threadIdx.x & 31;
     int lo = 0, hi = T;  // answer in [lo, hi)
     while (hi - lo > 1) {
-        int mid = (lo + hi) >> 1;
-        if (__ldg(off + mid) <= x) lo = mid; else hi = mid;
+        const int step = (hi - lo + 31) >> 5;
+        const int idx = lo + lane * step;
+        const bool le = idx < hi && __ldg(off + idx) <= x;
+        const unsigned m = __ballot_sync(0xffffffffu, le);  // offsets ascend: a prefix of the lanes
+        const int k = m ? 31 - __clz(m) : 0;
+        lo += k * step;
+        hi = (lo + step < hi) ? lo + step : hi;
     }
     return lo;
 }
