@@ -34,7 +34,6 @@ constexpr int kSelW = 16;          // binades in the fine window of round 1
 constexpr int kSelM = 7;           // log2(cells per binade) in the window
 constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
 constexpr int kMidN = 131072;      // tensors up to this size are solved start to finish by one CTA of their own
-constexpr int64_t kSelMinChunk = 98304;   // elements per flat streaming CTA, at least
 constexpr int kStageCap = 320;     // per-warp staging entries for compaction
 constexpr int kParkMax = 256;      // values one warp can park between two checks of round 2 (32 lanes x 8)
 constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
@@ -1824,14 +1823,12 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
         e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
     }
-    // Flat streaming CTAs (kSelResident are resident per SM): each pays a set-up, a flush of its cells
-    // and an arrival, so they get at least kSelMinChunk elements; between one and two waves, the more
-    // the better the balance against the per-tensor CTAs of the same grid.
+    // Flat streaming CTAs: one wave (kSelResident per SM).  Each CTA pays a set-up, a flush of its
+    // cells and an arrival per tensor piece, so larger chunks stream more of the time; a second wave
+    // balanced a lone call slightly better in round 1 but cost throughput whenever several calls
+    // (workers on their own streams) share the GPU.
     const int64_t wave = (int64_t)kSelResident * sm_count;
-    int64_t want = total / kSelMinChunk;
-    if (want < wave) want = wave;
-    if (want > 2 * wave) want = 2 * wave;
-    const int target = want < kMaxFlatCtas ? (int)want : kMaxFlatCtas;
+    const int target = wave < kMaxFlatCtas ? (int)wave : kMaxFlatCtas;
     FlatGrid g = make_flat_grid(total, target, 32768);
     SelArgs A;
     A.grad = d_grad; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
