@@ -285,7 +285,14 @@ k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* _
                 const int ng = (int)(g_full - g_beg);
                 const char* rows = reinterpret_cast<const char*>(&sh_lv[0][0]);
                 constexpr int kRow = (kMaxLevels + 1) * (int)sizeof(float);
+                constexpr int kAhead = 16;  // trips (of kWarps groups) between two prefetch requests
                 for (int gl = warp; gl < ng; gl += kWarps) {
+                    // every kAhead trips the first K threads ask L2 for the K workers' words of the
+                    // kAhead trips after the next kAhead (no gain at one bit per code)
+                    const int tr = gl / kWarps;
+                    if (BITS >= 2 && (tr & (kAhead - 1)) == 0 && (int)threadIdx.x < K && (tr + 2 * kAhead) * kWarps <= ng)
+                        prefetch_l2(sh_pk[threadIdx.x] + (g_beg + (int64_t)(tr + kAhead) * kWarps) * (4 * BITS),
+                                    kAhead * kWarps * 4u * BITS * 4u);
                     const int64_t wi = w0 + (int64_t)gl * (4 * BITS);
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
                     int k0 = 0;

@@ -75,6 +75,16 @@ __device__ __forceinline__ void for_each_piece(const int64_t* __restrict__ off, 
     }
 }
 
+// Asks L2 to fetch `bytes` (a multiple of 16) from a 16-byte aligned global address.  One thread of
+// a CTA issues it for the block the CTA will read a couple of loop trips later: the loads then find
+// their lines in L2, which keeps far more DRAM requests in flight than the registers of the loop can.
+// It pays in loops that compute for a while between loads (round 2 of the selection); loops that are
+// already bound by DRAM (BinGrad-b passes, the threshold quantizer) ran slower with it.
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(p), "r"(bytes) : "memory");
+}
+
 // Block-cooperative visit of grad[pb, pe): 128-bit loads on the aligned body,
 // scalar loads on the ragged head and tail.  f(float) is called once per element.
 template <class F>

@@ -364,6 +364,8 @@ __device__ __forceinline__ float max3f(float a, float b, float c)
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
+constexpr int kPrefetchTrips = 2;                         // how far ahead of the loads L2 is asked for a block
+constexpr uint32_t kTripBytes = 4u * kSelThreads * 16u;  // one trip of a CTA's streaming loop
 // shared-memory add without a return value, on a 32-bit shared address
 __device__ __forceinline__ void red_shared_add(uint32_t addr, uint32_t v)
 {
@@ -462,7 +464,10 @@ __device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     int64_t i = (a >> 2) + tid;
     const int64_t e = b >> 2;
+    int64_t pf = (a >> 2) + (int64_t)kPrefetchTrips * 4 * kSelThreads;
     for (; i + 3 * kSelThreads < e; i += 4 * kSelThreads) {
+        if (tid == 0 && pf + 4 * kSelThreads <= e) prefetch_l2(g4 + pf, kTripBytes);
+        pf += 4 * kSelThreads;
         float4 x[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i + u * kSelThreads);
@@ -520,7 +525,8 @@ __device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx,
 // Marks, in the space of raw fp32 bit patterns, every block of 2^17 patterns that can hold a value
 // whose key lies in one of the table's intervals (called by all threads).  A block of 2^17 aligned
 // keys is a block of 2^17 aligned patterns; -0 shares the block of the smallest negative values, and
-// with magnitude_only both signs of a pattern are marked.
+// with magnitude_only both signs of a pattern are marked.  Block b of a word sits at bit 31 - (b & 31):
+// a left shift by the block index brings its bit to the top of the word.
 __device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
 {
     for (int i = threadIdx.x; i < 1024; i += kSelThreads) tb.coarse[i] = 0u;
@@ -529,10 +535,10 @@ __device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
         const uint32_t ba = tb.klo[threadIdx.x] >> 17, bb = tb.khi[threadIdx.x] >> 17;
         for (uint32_t b = ba; b <= bb; ++b) {
             const uint32_t pblk = (b & 0x4000u) ? (b ^ 0x4000u) : (~b & 0x7fffu);
-            atomicOr(&tb.coarse[pblk >> 5], 1u << (pblk & 31));
+            atomicOr(&tb.coarse[pblk >> 5], 0x80000000u >> (pblk & 31));
             if (magnitude_only || pblk == 0u) {
                 const uint32_t twin = pblk ^ 0x4000u;
-                atomicOr(&tb.coarse[twin >> 5], 1u << (twin & 31));
+                atomicOr(&tb.coarse[twin >> 5], 0x80000000u >> (twin & 31));
             }
         }
     }
@@ -545,14 +551,38 @@ struct Round2Warp {
     uint32_t fillp;   // and their fill counter (bumped by the lanes that hit)
 
     // Phase A for one element: no warp collective, only the lanes that pass the bitmap test do work.
+    __device__ __forceinline__ void park(uint32_t bits)
+    {
+        const uint32_t pos = atom_shared_add(fillp, 1u);
+        asm volatile("st.shared.u32 [%0], %1;" :: "r"(stage + (pos << 2)), "r"(bits) : "memory");
+    }
+    __device__ __forceinline__ uint32_t top_is_hit(uint32_t bits) const
+    {
+        uint32_t word;
+        asm("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(coarse + ((bits >> 20) & 0xffcu)));
+        return __funnelshift_l(0u, word, bits >> 17);  // the block's bit is now bit 31
+    }
     __device__ __forceinline__ void one(float v)
     {
         const uint32_t bits = __float_as_uint(v);
-        uint32_t word;
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(coarse + ((bits >> 20) & 0xffcu)));
-        if (__funnelshift_r(word, 0u, bits >> 17) & 1u) {
-            const uint32_t pos = atom_shared_add(fillp, 1u);
-            asm volatile("st.shared.u32 [%0], %1;" :: "r"(stage + (pos << 2)), "r"(bits) : "memory");
+        if (top_is_hit(bits) >> 31) park(bits);
+    }
+    // Branch-free form for the main loop: shifts `hits` left and appends this element's bit.
+    __device__ __forceinline__ void test(float v, uint32_t& hits) const
+    {
+        hits = __funnelshift_l(top_is_hit(__float_as_uint(v)), hits, 1);
+    }
+    // Parks the elements marked in `hits` (bit 7 = the first of the eight elements tested: p[0].x,
+    // ..., p[0].w, p[stride].x, ...).  The values are read again, from L1: a hit is rare, and a
+    // register cannot be picked by a run-time index.
+    __device__ __forceinline__ void park_hits(uint32_t hits, const float4* p, int stride)
+    {
+        while (hits) {
+            const int b = 31 - __clz(hits);
+            hits &= ~(1u << b);
+            const int j = 7 - b;
+            const float* src = reinterpret_cast<const float*>(p + ((j & 4) ? stride : 0)) + (j & 3);
+            park(__float_as_uint(__ldg(src)));
         }
     }
 };
@@ -598,14 +628,22 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     const int64_t e = b >> 2;
     int64_t i0 = (a >> 2) + warp * 32;  // the trip counts below are warp-uniform
+    // Trips of 4 x kSelThreads float4 (one contiguous block of kTripBytes per CTA).  One thread asks
+    // L2 for the block kPrefetchTrips ahead, so that the loads below find their lines there.
+    int64_t pf = (a >> 2) + (int64_t)kPrefetchTrips * 4 * kSelThreads;
     for (; i0 + 3 * kSelThreads + 32 <= e; i0 += 4 * kSelThreads) {
+        if (threadIdx.x == 0 && pf + 4 * kSelThreads <= e) prefetch_l2(g4 + pf, kTripBytes);
+        pf += 4 * kSelThreads;
         float4 x[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i0 + lane + u * kSelThreads);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            w.one(x[u].x); w.one(x[u].y); w.one(x[u].z); w.one(x[u].w);
-            if (u & 1) check();
+        for (int h = 0; h < 4; h += 2) {
+            uint32_t hits = 0u;
+            w.test(x[h].x, hits); w.test(x[h].y, hits); w.test(x[h].z, hits); w.test(x[h].w, hits);
+            w.test(x[h + 1].x, hits); w.test(x[h + 1].y, hits); w.test(x[h + 1].z, hits); w.test(x[h + 1].w, hits);
+            if (hits) w.park_hits(hits, g4 + i0 + lane + h * kSelThreads, kSelThreads);
+            check();
         }
     }
     if (i0 < e) {
