@@ -790,6 +790,87 @@ __device__ __forceinline__ int find_new_interval(const SolverShared& S, uint32_t
     return (key >= S.niv[lo].klo && key <= S.niv[lo].khi) ? lo : -1;
 }
 
+// ---------------------------------------------------------------------------
+// Ascending bitonic sort of P keys in shared memory (P a power of two, at most 8 * kSelThreads),
+// called by all threads of the CTA; the keys are ordered on return (a barrier has been passed).
+// Compare-exchange distances of 256 and more are done by the whole CTA with a barrier per stage;
+// distances 8..128 stay inside an aligned block of 256 keys, which one warp owns and orders with
+// warp barriers only; distances 4, 2, 1 stay inside 8 consecutive keys, which one lane holds in
+// registers.  For 4096 keys that is 10 CTA barriers instead of 78.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void cmpx(uint32_t& a, uint32_t& b, bool up)
+{
+    const uint32_t lo = a < b ? a : b, hi = a < b ? b : a;
+    a = up ? lo : hi;
+    b = up ? hi : lo;
+}
+
+__device__ void block_bitonic_sort(uint32_t* keys, int P)
+{
+    if (P < 256) {  // few stages: the plain network
+        for (int k = 2; k <= P; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int i = threadIdx.x; i < P; i += kSelThreads) {
+                    const int ixj = i ^ j;
+                    if (ixj > i) {
+                        const uint32_t a = keys[i], b = keys[ixj];
+                        const bool up = (i & k) == 0;
+                        if ((a > b) == up) { keys[i] = b; keys[ixj] = a; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        return;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int k = 2; k <= P; k <<= 1) {
+        int j = k >> 1;
+        for (; j >= 256; j >>= 1) {  // CTA-wide stages
+            for (int q = threadIdx.x; q < (P >> 1); q += kSelThreads) {
+                const int i = ((q & ~(j - 1)) << 1) | (q & (j - 1));
+                uint32_t a = keys[i], b = keys[i | j];
+                cmpx(a, b, (i & k) == 0);
+                keys[i] = a; keys[i | j] = b;
+            }
+            __syncthreads();
+        }
+        for (int wb = warp * 256; wb < P; wb += kSelWarps * 256) {  // the 256-key blocks of this warp
+            uint32_t* blk = keys + wb;
+            int jj = j;
+            for (; jj >= 8; jj >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int q = lane + 32 * u;
+                    const int i = ((q & ~(jj - 1)) << 1) | (q & (jj - 1));
+                    uint32_t a = blk[i], b = blk[i | jj];
+                    cmpx(a, b, ((wb + i) & k) == 0);
+                    blk[i] = a; blk[i | jj] = b;
+                }
+                __syncwarp();
+            }
+            // distances 4, 2, 1 (those not above k / 2) on this lane's 8 consecutive keys
+            uint4* v4 = reinterpret_cast<uint4*>(blk + 8 * lane);
+            uint4 lo4 = v4[0], hi4 = v4[1];
+            uint32_t r[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+            const int i0 = wb + 8 * lane;
+#pragma unroll
+            for (int d = 4; d >= 1; d >>= 1) {
+                if (d <= jj) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if ((e & d) == 0) cmpx(r[e], r[e | d], ((i0 + e) & k) == 0);
+                }
+            }
+            v4[0] = make_uint4(r[0], r[1], r[2], r[3]);
+            v4[1] = make_uint4(r[4], r[5], r[6], r[7]);
+            __syncwarp();
+        }
+        // the next k starts with a CTA-wide stage only when k >= 256
+        if ((k << 1) >= 512 || k == P) __syncthreads();
+    }
+}
+
 // Sorting finish (ORQ): when the elements left inside the candidate intervals fit in shared
 // memory, they are sorted, run-length encoded into single-key cells with exact prefix counts
 // and sums, and one more solver pass resolves every open level at once.
@@ -806,42 +887,82 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     if (threadIdx.x == 0) S.n_keys = 0;
     if (threadIdx.x < kMaxIv) { S.ivstart[threadIdx.x] = 0; S.ivufirst[threadIdx.x] = -1; S.ivpre[threadIdx.x] = 0.0; }
     __syncthreads();
-    for (long long i0 = threadIdx.x; i0 < src_cnt; i0 += 4 * kSelThreads) {
-        uint32_t key[4];
-        bool ok[4];
+    // Filter of the copied keys: the lower and upper keys of the new intervals in two compact arrays
+    // (padded to 64 entries), a six-step search without branches, eight keys per thread in flight, and
+    // one shared counter update per warp and key column instead of one per accepted key.
+    __shared__ uint32_t f_lo[kMaxIv], f_hi[kMaxIv];
+    static_assert(kMaxIv == 64, "the search below takes six halving steps");
+    if (threadIdx.x < kMaxIv) {
+        const bool real = (int)threadIdx.x < S.nm;
+        f_lo[threadIdx.x] = real ? S.niv[threadIdx.x].klo : 0xffffffffu;  // no key has this value (NaN pattern)
+        f_hi[threadIdx.x] = real ? S.niv[threadIdx.x].khi : 0u;
+    }
+    __syncthreads();
+    OGQ_TICK(st, 10);
+    {
+        const int lane = threadIdx.x & 31;
+        constexpr int kCols = 8;
+        // the keys come from L2 (another SM wrote them): the loads of the next trip are issued before
+        // this trip's keys are searched, so that one round trip is hidden behind the other's work
+        auto fetch = [&](uint32_t* k, long long at) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {  // issue the loads together: they come from L2
-            const long long i = i0 + (long long)u * kSelThreads;
-            ok[u] = i < src_cnt;
-            key[u] = ok[u] ? __ldcg(buf + i) : 0u;
-        }
+            for (int u = 0; u < kCols; ++u) {
+                const long long i = at + u * 32 + lane;
+                k[u] = (i < src_cnt) ? __ldcg(buf + i) : 0u;
+            }
+        };
+        int top = 2;
+        while (top < S.nm) top <<= 1;
+        uint32_t nxt[kCols];
+        long long i0 = (long long)(threadIdx.x & ~31) * kCols;
+        if (i0 < src_cnt) fetch(nxt, i0);
+        for (; i0 < src_cnt; i0 += (long long)kCols * kSelThreads) {
+            uint32_t key[kCols];
+            bool in[kCols];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (ok[u] && find_new_interval(S, key[u]) >= 0) {
-                const int pos = atomicAdd(&S.n_keys, 1);
-                if (pos < kSmallN) skeys[pos] = key[u];
+            for (int u = 0; u < kCols; ++u) key[u] = nxt[u];
+            if (i0 + (long long)kCols * kSelThreads < src_cnt) fetch(nxt, i0 + (long long)kCols * kSelThreads);
+            int idx[kCols];
+#pragma unroll
+            for (int u = 0; u < kCols; ++u) idx[u] = 0;
+            // halving steps over the first `top` entries only (top = the power of two that covers the
+            // intervals): the table reads of 16 warps are what this loop is bound by
+            for (int step = top >> 1; step >= 1; step >>= 1) {
+#pragma unroll
+                for (int u = 0; u < kCols; ++u)
+                    if (f_lo[idx[u] + step] <= key[u]) idx[u] += step;
+            }
+            unsigned m[kCols];
+            int total = 0;
+#pragma unroll
+            for (int u = 0; u < kCols; ++u) {
+                in[u] = (i0 + u * 32 + lane < src_cnt) && key[u] >= f_lo[idx[u]] && key[u] <= f_hi[idx[u]];
+                m[u] = __ballot_sync(0xffffffffu, in[u]);
+                total += __popc(m[u]);
+            }
+            if (total) {  // one counter update per warp and trip
+                int pos = 0;
+                if (lane == 0) pos = atomicAdd(&S.n_keys, total);
+                pos = __shfl_sync(0xffffffffu, pos, 0);
+#pragma unroll
+                for (int u = 0; u < kCols; ++u) {
+                    const int at = pos + __popc(m[u] & ((1u << lane) - 1u));
+                    if (in[u] && at < kSmallN) skeys[at] = key[u];
+                    pos += __popc(m[u]);
+                }
             }
         }
     }
+    OGQ_TICK(st, 11);
     __syncthreads();
     const int c = S.n_keys < kSmallN ? S.n_keys : kSmallN;
     int P = 1;
     while (P < c) P <<= 1;
+    OGQ_TICK(st, 6);
     for (int i = c + threadIdx.x; i < kSmallN; i += kSelThreads) skeys[i] = 0xffffffffu;
     __syncthreads();
-    for (int k = 2; k <= P; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < P; i += kSelThreads) {
-                const int ixj = i ^ j;
-                if (ixj > i) {
-                    const uint32_t a = skeys[i], b = skeys[ixj];
-                    const bool up = (i & k) == 0;
-                    if ((a > b) == up) { skeys[i] = b; skeys[ixj] = a; }
-                }
-            }
-            __syncthreads();
-        }
-    }
+    block_bitonic_sort(skeys, P);
+    OGQ_TICK(st, 7);
     // pass 1: run starts and value sums of this thread's kPer consecutive sorted elements
     const int base = threadIdx.x * kPer;
     uint32_t k[kPer];
@@ -862,6 +983,7 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     double sbase = ls, tsum;
     block_excl_scan(ubase, sbase, S.sc, S.ss, tu, tsum);
     if (threadIdx.x == 0) S.n_unique = (int)tu;
+    OGQ_TICK(st, 8);
     // pass 2: first element of every interval
     {
         int nf = 0;
@@ -939,6 +1061,7 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
         sel_init_slots(S.view);
         S.internal = (S.n_keys > kSmallN) ? 1 : 0;
     }
+    OGQ_TICK(st, 9);
     // one thread per level, one depth at a time (every cell is a single key now, so each solve is exact)
     for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
         __syncthreads();
@@ -1393,20 +1516,7 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
         keys[i] = key;
     }
     __syncthreads();
-    // bitonic sort, ascending
-    for (int k = 2; k <= P; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < P; i += kSelThreads) {
-                const int ixj = i ^ j;
-                if (ixj > i) {
-                    const uint32_t a = keys[i], b = keys[ixj];
-                    const bool up = (i & k) == 0;
-                    if ((a > b) == up) { keys[i] = b; keys[ixj] = a; }
-                }
-            }
-            __syncthreads();
-        }
-    }
+    block_bitonic_sort(keys, P);  // ascending
     int stbits = 0;
     if (sh_flag) {
         if (threadIdx.x == 0) {

@@ -192,3 +192,45 @@ def test_flat_tensor_with_crowded_cells():
     db = DeviceBucket(v, off)
     lv, st = db.levels_orq(9)
     assert st[0] & ogq.OGQ_ST_NONFINITE
+
+
+def test_resnet50_eight_workers_on_eight_streams():
+    """The benchmark's launch configuration: K = 8 workers, each on a CUDA stream and a scratch buffer
+    of its own, all in flight together.  Every worker's levels and packed words must equal what the
+    same calls give one after the other on one stream (the kernels are bit-reproducible and share
+    nothing between calls), and worker 0's levels must equal the oracle's."""
+    K, s = 8, 9
+    b = wl.resnet50_bucket(0)
+    db = DeviceBucket(b.values, b.offsets)
+    bits = ogq.ogq_bits_for_levels(s)
+    h_po = ogq.ogq_packed_layout(db.h_off, bits)
+    po = torch.from_numpy(h_po).to(db.dev)
+    grads = worker_variants(db, K)
+
+    def run(streams):
+        lvs, pks, sts = [], [], []
+        wss = [torch.empty(db.ws_bytes, dtype=torch.uint8, device=db.dev) for _ in range(K)]
+        torch.cuda.synchronize()
+        for k in range(K):
+            lv = torch.zeros((db.T, s), device=db.dev)
+            st = torch.zeros(db.T, dtype=torch.int32, device=db.dev)
+            pk = torch.zeros(int(h_po[-1]), dtype=torch.int32, device=db.dev)
+            lvs.append(lv); pks.append(pk); sts.append(st)
+        torch.cuda.synchronize()
+        for k in range(K):
+            stream = streams[k] if streams else None
+            ctx = torch.cuda.stream(stream) if stream is not None else torch.cuda.stream(torch.cuda.current_stream())
+            with ctx:
+                ogq.ogq_levels_orq(grads[k], db.off, db.T, db.N, s, lvs[k], sts[k], wss[k], db.ws_bytes, stream)
+                ogq.ogq_quantize_pack(grads[k], db.off, db.T, db.N, ogq.OGQ_ORQ, s, lvs[k], None, 5, k, po, pks[k], stream)
+        torch.cuda.synchronize()
+        return [l.cpu().numpy() for l in lvs], [p.cpu().numpy() for p in pks], [x.cpu().numpy() for x in sts]
+
+    serial = run(None)
+    together = run([torch.cuda.Stream(device=db.dev) for _ in range(K)])
+    for k in range(K):
+        assert not np.any(together[2][k] & (ogq.OGQ_ST_INTERNAL | ogq.OGQ_ST_ITER_CAP | ogq.OGQ_ST_NONFINITE))
+        assert np.array_equal(serial[0][k], together[0][k]), k
+        assert np.array_equal(serial[1][k], together[1][k]), k
+    want, _ = oracle.bucket_levels_orq(b.values, b.offsets, s)
+    assert levels_close(together[0][0], want)
