@@ -286,41 +286,49 @@ k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* _
                 const char* rows = reinterpret_cast<const char*>(&sh_lv[0][0]);
                 constexpr int kRow = (kMaxLevels + 1) * (int)sizeof(float);
                 constexpr int kAhead = 16;  // trips (of kWarps groups) between two prefetch requests
-                for (int gl = warp; gl < ng; gl += kWarps) {
+                // adds the levels of the four codes of this lane in word w (worker row r) to a[0..3]
+                auto add4 = [&](uint32_t w, const char* r, float* a) {
+                    const uint32_t f = (w >> shift) << 2;  // byte offsets of the 4 codes
+                    a[0] = __fadd_rn(a[0], *reinterpret_cast<const float*>(r + (f & (kMask1 << 2))));
+                    a[1] = __fadd_rn(a[1], *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2))));
+                    a[2] = __fadd_rn(a[2], *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2))));
+                    a[3] = __fadd_rn(a[3], *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2))));
+                };
+                // two groups per warp and trip: sixteen word loads in flight per lane
+                for (int gl = warp; gl < ng; gl += 2 * kWarps) {
                     // every kAhead trips the first K threads ask L2 for the K workers' words of the
                     // kAhead trips after the next kAhead (no gain at one bit per code)
                     const int tr = gl / kWarps;
                     if (BITS >= 2 && (tr & (kAhead - 1)) == 0 && (int)threadIdx.x < K && (tr + 2 * kAhead) * kWarps <= ng)
                         prefetch_l2(sh_pk[threadIdx.x] + (g_beg + (int64_t)(tr + kAhead) * kWarps) * (4 * BITS),
                                     kAhead * kWarps * 4u * BITS * 4u);
-                    const int64_t wi = w0 + (int64_t)gl * (4 * BITS);
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                    const bool two = gl + kWarps < ng;
+                    const int64_t wa = w0 + (int64_t)gl * (4 * BITS);
+                    const int64_t wb = two ? wa + (int64_t)kWarps * (4 * BITS) : wa;
+                    float a[4] = {0.f, 0.f, 0.f, 0.f}, b[4] = {0.f, 0.f, 0.f, 0.f};
                     int k0 = 0;
                     for (; k0 + 8 <= K; k0 += 8) {
-                        uint32_t w[8];
+                        uint32_t xa[8], xb[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) w[u] = __ldg(sh_pk[k0 + u] + wi);
+                        for (int u = 0; u < 8; ++u) xa[u] = __ldg(sh_pk[k0 + u] + wa);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) xb[u] = __ldg(sh_pk[k0 + u] + wb);
                         const char* r0 = rows + k0 * kRow;
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const uint32_t f = (w[u] >> shift) << 2;  // byte offsets of the 4 codes
-                            const char* r = r0 + u * kRow;
-                            a0 = __fadd_rn(a0, *reinterpret_cast<const float*>(r + (f & (kMask1 << 2))));
-                            a1 = __fadd_rn(a1, *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2))));
-                            a2 = __fadd_rn(a2, *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2))));
-                            a3 = __fadd_rn(a3, *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2))));
-                        }
+                        for (int u = 0; u < 8; ++u) add4(xa[u], r0 + u * kRow, a);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) add4(xb[u], r0 + u * kRow, b);
                     }
                     for (; k0 < K; ++k0) {
-                        const uint32_t f = (__ldg(sh_pk[k0] + wi) >> shift) << 2;
-                        const char* r = rows + k0 * kRow;
-                        a0 = __fadd_rn(a0, *reinterpret_cast<const float*>(r + (f & (kMask1 << 2))));
-                        a1 = __fadd_rn(a1, *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2))));
-                        a2 = __fadd_rn(a2, *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2))));
-                        a3 = __fadd_rn(a3, *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2))));
+                        const uint32_t xa = __ldg(sh_pk[k0] + wa), xb = __ldg(sh_pk[k0] + wb);
+                        add4(xa, rows + k0 * kRow, a);
+                        add4(xb, rows + k0 * kRow, b);
                     }
-                    dst4[(size_t)gl * 32] = make_float4(__fmul_rn(a0, scale), __fmul_rn(a1, scale),
-                                                        __fmul_rn(a2, scale), __fmul_rn(a3, scale));
+                    dst4[(size_t)gl * 32] = make_float4(__fmul_rn(a[0], scale), __fmul_rn(a[1], scale),
+                                                        __fmul_rn(a[2], scale), __fmul_rn(a[3], scale));
+                    if (two)
+                        dst4[(size_t)(gl + kWarps) * 32] = make_float4(__fmul_rn(b[0], scale), __fmul_rn(b[1], scale),
+                                                                       __fmul_rn(b[2], scale), __fmul_rn(b[3], scale));
                 }
             }
         }
