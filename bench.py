@@ -352,7 +352,7 @@ def run_ours(args):
     # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from one ncu
     # capture of the current kernels on a 2^26-element tensor with s = 9; traffic grows in proportion to
     # the elements streamed, so a full launch is this figure times N.  Other schemes: not captured.
-    ncu_dram_bytes_per_element = {"k_sel_round1": 4.466, "k_sel_round2": 4.274, "k_quantize_pack_random": 4.394}
+    ncu_dram_bytes_per_element = {"k_sel_round1": 4.461, "k_sel_round2": 4.232, "k_quantize_pack_random": 4.397}
     traffic = None
     if args.scheme == "orq9" and dom in ncu_dram_bytes_per_element:
         traffic = ncu_dram_bytes_per_element[dom] * N
