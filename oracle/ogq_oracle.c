@@ -5,7 +5,9 @@
  * of "Optimal Gradient Quantization Condition for Communication-Efficient
  * Distributed Training" computes: per-tensor level solvers for BinGrad-b,
  * BinGrad-pb and ORQ, the three quantizers, a bit-packing format and the
- * decode-and-sum step.  Arithmetic is fp64 (sums in long double) on fp32
+ * decode-and-sum step; then gradient clipping, an entropy-dense (base-s) wire
+ * format, the quantization error and refinement sweeps over the greedy ORQ
+ * levels.  Arithmetic is fp64 (sums in long double) on fp32
  * inputs, except the one rounding decision that is defined in fp32 (see
  * ogq_oracle_quantize).  It shares no code with the CUDA library and is only
  * called from the tests, the smoke check and the benchmark's CPU baseline.
@@ -401,4 +403,196 @@ void ogq_oracle_unpack_sum(const uint32_t *const *packed, const float *const *le
         }
         out[i] = (float)((double)scale * acc);
     }
+}
+
+/* ======================================================================== */
+/* Extensions beyond the per-tensor core: gradient clipping, an entropy-     */
+/* dense wire format, the quantization error and a refinement of the greedy  */
+/* ORQ levels.                                                                */
+/* ======================================================================== */
+
+/* ------------------------------------------------------------------------ */
+/* Gradient clipping (Section "Experiments", paragraph after the list of     */
+/* methods): clip(v) = sign(v) * min(|v|, c * sigma), sigma^2 the variance   */
+/* of the gradient being quantized (here: of the tensor or bucket), c = 2.5  */
+/* in the ImageNet runs and 1.7 or 2.5 in the clipping table.  The variance  */
+/* is taken about the mean, over all n elements (1/n).  The threshold is     */
+/* rounded to fp32 because clipped elements take exactly that value.         */
+/* Returns status bits; tau = 0 for an empty tensor.                         */
+/* ------------------------------------------------------------------------ */
+int ogq_oracle_clip_threshold(const float *v, int64_t n, double c, float *tau)
+{
+    *tau = 0.0f;
+    if (n <= 0) return OGQ_ST_EMPTY;
+    long double s = 0.0L;
+    for (int64_t i = 0; i < n; ++i) {
+        if (!isfinite((double)v[i])) return OGQ_ST_NONFINITE;
+        s += (long double)v[i];
+    }
+    long double mean = s / (long double)n;
+    long double q = 0.0L;
+    for (int64_t i = 0; i < n; ++i) {
+        long double d = (long double)v[i] - mean;
+        q += d * d;
+    }
+    double sigma = sqrt((double)(q / (long double)n));
+    *tau = (float)(c * sigma);
+    return 0;
+}
+
+void ogq_oracle_clip(const float *v, int64_t n, float tau, float *out)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float a = fabsf(v[i]);
+        float m = a < tau ? a : tau;
+        out[i] = v[i] < 0.0f ? -m : m;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Entropy-dense packing.  The compression ratios the paper quotes (x20.2    */
+/* for 3 levels, x13.8 for 5, x10.1 for 9) are 32 / log2(s): they assume     */
+/* that a code costs log2(s) bits, not ceil(log2 s).  The format here gets   */
+/* close to that with whole words: m consecutive codes are the base-s digits */
+/* of one 32-bit word, least significant digit first, m the largest count    */
+/* with s^m <= 2^32 (s = 3: 20 codes per word, 5: 13, 9: 10, 17: 7, 2: 32).  */
+/* Per tensor: word j = sum_{q<m} code[j*m + q] * s^q, missing codes of the  */
+/* last word are 0, and the region is zero padded to a multiple of 4 words.  */
+/* ------------------------------------------------------------------------ */
+int ogq_oracle_dense_digits(int s)
+{
+    if (s < 2) return 0;
+    int m = 0;
+    uint64_t p = 1;
+    while (p * (uint64_t)s <= ((uint64_t)1 << 32)) {
+        p *= (uint64_t)s;
+        ++m;
+    }
+    return m;
+}
+
+int64_t ogq_oracle_dense_words(int64_t n, int s)
+{
+    int m = ogq_oracle_dense_digits(s);
+    int64_t w = (n + m - 1) / m;
+    return (w + 3) / 4 * 4;
+}
+
+void ogq_oracle_pack_dense(const uint8_t *codes, int64_t n, int s, uint32_t *words)
+{
+    int m = ogq_oracle_dense_digits(s);
+    int64_t nw = ogq_oracle_dense_words(n, s);
+    memset(words, 0, (size_t)nw * sizeof(uint32_t));
+    for (int64_t j = 0; j * m < n; ++j) {
+        uint64_t w = 0, p = 1;
+        for (int q = 0; q < m; ++q) {
+            int64_t i = j * m + q;
+            if (i < n) w += (uint64_t)codes[i] * p;
+            p *= (uint64_t)s;
+        }
+        words[j] = (uint32_t)w;
+    }
+}
+
+void ogq_oracle_unpack_dense(const uint32_t *words, int64_t n, int s, uint8_t *codes)
+{
+    int m = ogq_oracle_dense_digits(s);
+    for (int64_t i = 0; i < n; ++i) {
+        uint64_t w = words[i / m];
+        for (int q = 0; q < (int)(i % m); ++q) w /= (uint64_t)s;
+        codes[i] = (uint8_t)(w % (uint64_t)s);
+    }
+}
+
+void ogq_oracle_unpack_sum_dense(const uint32_t *const *packed, const float *const *levels, int K,
+                                 int64_t n, int s, float scale, float *out)
+{
+    int m = ogq_oracle_dense_digits(s);
+    for (int64_t i = 0; i < n; ++i) {
+        double acc = 0.0;
+        for (int k = 0; k < K; ++k) {
+            uint64_t w = packed[k][i / m];
+            for (int q = 0; q < (int)(i % m); ++q) w /= (uint64_t)s;
+            acc += (double)levels[k][w % (uint64_t)s];
+        }
+        out[i] = (float)((double)scale * acc);
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Quantization error (the quantity tracked in the training-curve figure,    */
+/* ||Q(G) - G||^2).                                                           */
+/*   ogq_oracle_quant_error:    the realised error of given codes,           */
+/*       sum_i (levels[code_i] - v_i)^2.                                      */
+/*   ogq_oracle_expected_error: its expectation over the random rounding,    */
+/*       the functional the optimal condition minimises (proof of Theorem    */
+/*       1): sum_i (v_i - lo_i)(hi_i - v_i) with lo, hi the levels around    */
+/*       v_i; a value outside [b_0, b_{s-1}] is clipped to the end level and */
+/*       contributes (v_i - b_end)^2.                                         */
+/* ------------------------------------------------------------------------ */
+double ogq_oracle_quant_error(const float *v, int64_t n, const float *levels, const uint8_t *codes)
+{
+    long double e = 0.0L;
+    for (int64_t i = 0; i < n; ++i) {
+        long double d = (long double)levels[codes[i]] - (long double)v[i];
+        e += d * d;
+    }
+    return (double)e;
+}
+
+double ogq_oracle_expected_error(const float *v, int64_t n, int s, const float *levels)
+{
+    long double e = 0.0L;
+    for (int64_t i = 0; i < n; ++i) {
+        double x = (double)v[i];
+        double b0 = (double)levels[0], bs = (double)levels[s - 1];
+        if (x < b0) {
+            e += (long double)((b0 - x) * (b0 - x));
+            continue;
+        }
+        if (x > bs) {
+            e += (long double)((x - bs) * (x - bs));
+            continue;
+        }
+        int k = 0;
+        for (int q = 0; q < s; ++q) k += ((double)levels[q] <= x);
+        if (k < 1) k = 1;
+        if (k > s - 1) k = s - 1;
+        double lo = (double)levels[k - 1], hi = (double)levels[k];
+        e += (long double)((x - lo) * (hi - x));
+    }
+    return (double)e;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Beyond the greedy levels (the conclusion names the greedy algorithm as    */
+/* the part that may be improved).  Algorithm 1 fixes a level once it has    */
+/* been solved from its two brackets, so afterwards only the deepest levels  */
+/* satisfy the optimal condition against their final neighbours.  One        */
+/* refinement sweep re-solves every interior level in ascending order from   */
+/* its two current neighbours, b_k <- Q*(b_{k-1}, b_{k+1}), each update      */
+/* using the levels already updated in this sweep.  Q* is the exact          */
+/* minimiser of the expected error in b_k with the other levels held fixed,  */
+/* so no sweep increases the error.  Sweeps stop when one changes nothing    */
+/* (every level then satisfies the discrete condition against its final      */
+/* neighbours) or after max_sweeps.  levels: s values, ascending, in and out;*/
+/* the end levels stay.  Returns the number of sweeps that changed a level.  */
+/* ------------------------------------------------------------------------ */
+int ogq_oracle_refine_orq(const float *v, int64_t n, int s, float *levels, int max_sweeps)
+{
+    int changed_sweeps = 0;
+    if (n <= 0) return 0;
+    for (int it = 0; it < max_sweeps; ++it) {
+        int changed = 0;
+        for (int k = 1; k < s - 1; ++k) {
+            float nb = (float)ogq_oracle_qstar(v, n, (double)levels[k - 1], (double)levels[k + 1]);
+            if (nb != levels[k]) {
+                levels[k] = nb;
+                changed = 1;
+            }
+        }
+        if (!changed) break;
+        ++changed_sweeps;
+    }
+    return changed_sweeps;
 }

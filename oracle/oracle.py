@@ -70,6 +70,29 @@ def lib() -> ctypes.CDLL:
             ctypes.c_float, fp,
         ]
         L.ogq_oracle_unpack_sum.restype = None
+        L.ogq_oracle_clip_threshold.argtypes = [fp, i64, ctypes.c_double, fp]
+        L.ogq_oracle_clip_threshold.restype = ctypes.c_int
+        L.ogq_oracle_clip.argtypes = [fp, i64, ctypes.c_float, fp]
+        L.ogq_oracle_clip.restype = None
+        L.ogq_oracle_dense_digits.argtypes = [ctypes.c_int]
+        L.ogq_oracle_dense_digits.restype = ctypes.c_int
+        L.ogq_oracle_dense_words.argtypes = [i64, ctypes.c_int]
+        L.ogq_oracle_dense_words.restype = i64
+        L.ogq_oracle_pack_dense.argtypes = [u8, i64, ctypes.c_int, u32]
+        L.ogq_oracle_pack_dense.restype = None
+        L.ogq_oracle_unpack_dense.argtypes = [u32, i64, ctypes.c_int, u8]
+        L.ogq_oracle_unpack_dense.restype = None
+        L.ogq_oracle_unpack_sum_dense.argtypes = [
+            ctypes.POINTER(u32), ctypes.POINTER(fp), ctypes.c_int, i64, ctypes.c_int,
+            ctypes.c_float, fp,
+        ]
+        L.ogq_oracle_unpack_sum_dense.restype = None
+        L.ogq_oracle_quant_error.argtypes = [fp, i64, fp, u8]
+        L.ogq_oracle_quant_error.restype = ctypes.c_double
+        L.ogq_oracle_expected_error.argtypes = [fp, i64, ctypes.c_int, fp]
+        L.ogq_oracle_expected_error.restype = ctypes.c_double
+        L.ogq_oracle_refine_orq.argtypes = [fp, i64, ctypes.c_int, fp, ctypes.c_int]
+        L.ogq_oracle_refine_orq.restype = ctypes.c_int
     return _lib
 
 
@@ -177,7 +200,129 @@ def unpack_sum(packed: Sequence[np.ndarray], levels: Sequence[np.ndarray], n: in
     return out
 
 
+def clip_threshold(v, c: float) -> Tuple[np.float32, int]:
+    """tau = fp32(c * sigma), sigma^2 the variance of v about its mean (1/n)."""
+    v = _f32(v)
+    tau = ctypes.c_float(0.0)
+    st = lib().ogq_oracle_clip_threshold(_ptr(v, ctypes.c_float), v.size, float(c), ctypes.byref(tau))
+    return np.float32(tau.value), st
+
+
+def clip(v, tau: float) -> np.ndarray:
+    """sign(v) * min(|v|, tau), element by element."""
+    v = _f32(v)
+    out = np.zeros_like(v)
+    lib().ogq_oracle_clip(_ptr(v, ctypes.c_float), v.size, ctypes.c_float(float(tau)), _ptr(out, ctypes.c_float))
+    return out
+
+
+def dense_digits(s: int) -> int:
+    return int(lib().ogq_oracle_dense_digits(int(s)))
+
+
+def dense_words(n: int, s: int) -> int:
+    return int(lib().ogq_oracle_dense_words(int(n), int(s)))
+
+
+def pack_dense(codes, s: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    words = np.zeros(dense_words(codes.size, s), dtype=np.uint32)
+    lib().ogq_oracle_pack_dense(_ptr(codes, ctypes.c_uint8), codes.size, int(s), _ptr(words, ctypes.c_uint32))
+    return words
+
+
+def unpack_dense(words, n: int, s: int) -> np.ndarray:
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    codes = np.zeros(n, dtype=np.uint8)
+    lib().ogq_oracle_unpack_dense(_ptr(words, ctypes.c_uint32), int(n), int(s), _ptr(codes, ctypes.c_uint8))
+    return codes
+
+
+def unpack_sum_dense(packed: Sequence[np.ndarray], levels: Sequence[np.ndarray], n: int, s: int, scale: float) -> np.ndarray:
+    K = len(packed)
+    pk = [np.ascontiguousarray(p, dtype=np.uint32) for p in packed]
+    lv = [_f32(l) for l in levels]
+    pp = (ctypes.POINTER(ctypes.c_uint32) * K)(*[_ptr(p, ctypes.c_uint32) for p in pk])
+    lp = (ctypes.POINTER(ctypes.c_float) * K)(*[_ptr(l, ctypes.c_float) for l in lv])
+    out = np.zeros(n, dtype=np.float32)
+    lib().ogq_oracle_unpack_sum_dense(pp, lp, K, int(n), int(s), ctypes.c_float(float(scale)), _ptr(out, ctypes.c_float))
+    return out
+
+
+def quant_error(v, levels, codes) -> float:
+    """sum_i (levels[code_i] - v_i)^2."""
+    v = _f32(v)
+    lv = _f32(levels)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    return float(lib().ogq_oracle_quant_error(_ptr(v, ctypes.c_float), v.size, _ptr(lv, ctypes.c_float),
+                                              _ptr(codes, ctypes.c_uint8)))
+
+
+def expected_error(v, levels) -> float:
+    """Expectation of the random-rounding error over the draws: sum_i (v_i - lo_i)(hi_i - v_i)."""
+    v = _f32(v)
+    lv = _f32(levels)
+    return float(lib().ogq_oracle_expected_error(_ptr(v, ctypes.c_float), v.size, lv.size, _ptr(lv, ctypes.c_float)))
+
+
+def refine_orq(v, levels, max_sweeps: int) -> Tuple[np.ndarray, int]:
+    """Refinement sweeps b_k <- Q*(b_{k-1}, b_{k+1}) over the interior levels; returns (levels, sweeps that changed something)."""
+    v = _f32(v)
+    lv = _f32(levels).copy()
+    n = lib().ogq_oracle_refine_orq(_ptr(v, ctypes.c_float), v.size, lv.size, _ptr(lv, ctypes.c_float), int(max_sweeps))
+    return lv, int(n)
+
+
 # ---------------------------------------------------------------- per bucket
+
+
+def dense_layout(offsets, s: int) -> np.ndarray:
+    """Word offset of every tensor's region in the base-s format."""
+    offsets = np.asarray(offsets, dtype=np.int64)
+    T = offsets.size - 1
+    po = np.zeros(T + 1, dtype=np.int64)
+    for t in range(T):
+        po[t + 1] = po[t] + dense_words(int(offsets[t + 1] - offsets[t]), s)
+    return po
+
+
+def bucket_clip_thresholds(values, offsets, c: float) -> Tuple[np.ndarray, np.ndarray]:
+    offsets = np.asarray(offsets, dtype=np.int64)
+    T = offsets.size - 1
+    tau = np.zeros(T, dtype=np.float32)
+    st = np.zeros(T, dtype=np.int32)
+    for t in range(T):
+        tau[t], st[t] = clip_threshold(values[offsets[t] : offsets[t + 1]], c)
+    return tau, st
+
+
+def bucket_clip(values, offsets, tau) -> np.ndarray:
+    offsets = np.asarray(offsets, dtype=np.int64)
+    out = np.array(values, dtype=np.float32, copy=True)
+    for t in range(offsets.size - 1):
+        out[offsets[t] : offsets[t + 1]] = clip(values[offsets[t] : offsets[t + 1]], float(tau[t]))
+    return out
+
+
+def bucket_pack_dense(codes_per_tensor: Sequence[np.ndarray], offsets, s: int) -> Tuple[np.ndarray, np.ndarray]:
+    po = dense_layout(offsets, s)
+    out = np.zeros(int(po[-1]), dtype=np.uint32)
+    for t, codes in enumerate(codes_per_tensor):
+        out[po[t] : po[t + 1]] = pack_dense(codes, s)
+    return out, po
+
+
+def bucket_unpack_sum_dense(packed_k: Sequence[np.ndarray], levels_k: Sequence[np.ndarray], offsets, s: int, scale: float) -> np.ndarray:
+    offsets = np.asarray(offsets, dtype=np.int64)
+    T = offsets.size - 1
+    po = dense_layout(offsets, s)
+    out = np.zeros(int(offsets[-1]), dtype=np.float32)
+    for t in range(T):
+        n = int(offsets[t + 1] - offsets[t])
+        out[offsets[t] : offsets[t + 1]] = unpack_sum_dense(
+            [p[po[t] : po[t + 1]] for p in packed_k], [l[t] for l in levels_k], n, s, scale
+        )
+    return out
 
 
 def packed_layout(offsets, bits: int) -> np.ndarray:
