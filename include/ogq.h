@@ -23,6 +23,9 @@
  *     the data are reported per tensor in d_status (bits OGQ_ST_*), never by a
  *     trap.  There is no CPU fallback.
  *   - Levels are fp32 because they are what a worker sends next to its codes.
+ *   - Size limit of the selection solvers (ogq_levels_orq, ogq_levels_bingrad with
+ *     OGQ_BINGRAD_PB): total_elems below 2^32, because they count a tensor's elements in
+ *     32-bit cells; larger buckets return OGQ_ERR_UNSUPPORTED and enqueue nothing.
  */
 #ifndef OGQ_H_
 #define OGQ_H_
@@ -114,6 +117,9 @@ ogq_status ogq_levels_bingrad(const float *d_grad, const int64_t *d_off, int T, 
  *     before its kernels run, so leftovers of earlier calls do no harm, but two calls whose
  *     work overlaps on the GPU (different streams, no ordering between them) race on it and
  *     give wrong levels.  Order such calls, or use ogq_levels_bingrad with separate scratch.
+ *   - OGQ_ERR_LIMIT comes only from the tensor-count check above; a failing CUDA call is
+ *     OGQ_ERR_CUDA.  Host threads may make the first call on a device concurrently (the
+ *     address lookup is idempotent and its result is stored atomically).
  */
 #define OGQ_NOALLOC_MAX_TENSORS 1024
 ogq_status ogq_levels_bingrad_b_noalloc(const float *d_grad, const int64_t *d_off, int T,
@@ -126,7 +132,11 @@ ogq_status ogq_levels_bingrad_b_noalloc(const float *d_grad, const int64_t *d_of
  * maximum (Corollary 1); every other level is the middle of its two bracket
  * levels L < R: with T = sum_{L <= v <= R} (v - L) / (R - L), it is the
  * (floor(T) + 1)-th largest element of {L <= v <= R}, so every level is one of
- * the tensor's own values and the result is exact.
+ * the tensor's own values, found by exact selection (no sampling, no
+ * approximation of ranks).  T itself is evaluated in fp64 from exact integer
+ * partial sums; where T lies within fp64 rounding of an integer, the data value
+ * next to the one a higher-precision evaluation picks may be returned (both
+ * then satisfy the condition to rounding).
  * Output: d_levels [T][s] ascending, d_status [T].
  */
 ogq_status ogq_levels_orq(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems, int s,

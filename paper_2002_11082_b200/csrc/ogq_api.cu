@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 #include <string.h>
 
+#include <atomic>
 #include <vector>
 
 #include "../../include/ogq.h"
@@ -17,11 +18,11 @@ struct ProfRec {
 };
 static std::vector<ProfRec> g_prof;
 static bool g_prof_on = false;
-static unsigned long long g_launches = 0;
+static std::atomic<unsigned long long> g_launches{0};  // data-path calls may come from several host threads
 
 void launch_begin(const char* name, cudaStream_t stream)
 {
-    ++g_launches;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     if (!g_prof_on) return;
     ProfRec r;
     r.name = name;
@@ -52,13 +53,16 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 bool valid_orq_levels(int s) { return s == 3 || s == 5 || s == 9 || s == 17; }
 
+// The selection solvers count the elements of a tensor in 32-bit cells.
+bool select_size_ok(int64_t total_elems) { return total_elems < ((int64_t)1 << 32); }
+
 }  // namespace
 
 extern "C" {
 
 const char* ogq_version(void) { return "ogq 0.1 (sm_100a)"; }
 
-unsigned long long ogq_launch_count(void) { return ogq::g_launches; }
+unsigned long long ogq_launch_count(void) { return ogq::g_launches.load(std::memory_order_relaxed); }
 
 int ogq_profile_enable(int on)
 {
@@ -128,6 +132,7 @@ ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, 
         lloyd_iters > 1024)
         return OGQ_ERR_INVALID_ARG;
     if (variant != OGQ_BINGRAD_PB && variant != OGQ_BINGRAD_B) return OGQ_ERR_UNSUPPORTED;
+    if (variant == OGQ_BINGRAD_PB && !select_size_ok(total_elems)) return OGQ_ERR_UNSUPPORTED;
     if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
     if (variant == OGQ_BINGRAD_B && !d_thresh) return OGQ_ERR_INVALID_ARG;
     if (T == 0) return OGQ_OK;
@@ -161,7 +166,6 @@ ogq_status ogq_levels_bingrad_b_noalloc(const float* d_grad, const int64_t* d_of
     if (sms <= 0) return OGQ_ERR_CUDA;
     cudaError_t e = ogq::launch_levels_bingrad_b_static(d_grad, d_off, T, total_elems, lloyd_iters, d_levels,
                                                         d_thresh, d_status, sms, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return OGQ_ERR_LIMIT;
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 
@@ -170,7 +174,7 @@ ogq_status ogq_levels_orq(const float* d_grad, const int64_t* d_off, int T, int6
                           ogq_stream_t stream)
 {
     if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_status) return OGQ_ERR_INVALID_ARG;
-    if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
+    if (!valid_orq_levels(s) || !select_size_ok(total_elems)) return OGQ_ERR_UNSUPPORTED;
     if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
     if (T == 0) return OGQ_OK;
     if (!d_ws || ((uintptr_t)d_ws & 255u)) return OGQ_ERR_WORKSPACE;

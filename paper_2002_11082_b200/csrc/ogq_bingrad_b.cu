@@ -8,6 +8,8 @@
 // order by the last CTA to arrive, so results do not depend on scheduling.
 #include <math.h>
 
+#include <atomic>
+
 #include "ogq_common.cuh"
 #include "ogq_internal.h"
 #include "ogq_ws.h"
@@ -162,7 +164,9 @@ static __device__ __align__(256) unsigned char g_bb_static_scratch[kNoAllocBytes
 
 // Device address of the array above, looked up once per device.  In host code the symbol's name is
 // only a handle, not an address the GPU can use, so the address has to come from the runtime.
-static void* g_bb_static_ptr[kNoAllocMaxDevices] = {nullptr};
+// Two host threads that make the first call on a device at the same time both look the address up and
+// store the same value: the slot is atomic so that this is well defined.
+static std::atomic<void*> g_bb_static_ptr[kNoAllocMaxDevices];
 
 cudaError_t launch_levels_bingrad_b_static(const float* d_grad, const int64_t* d_off, int T, int64_t total,
                                            int lloyd_iters, float* d_levels, float* d_thresh,
@@ -172,18 +176,20 @@ cudaError_t launch_levels_bingrad_b_static(const float* d_grad, const int64_t* d
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kNoAllocMaxDevices) return cudaErrorInvalidDevice;
-    if (g_bb_static_ptr[dev] == nullptr) {
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_bb_static_scratch);
+    void* scratch = g_bb_static_ptr[dev].load(std::memory_order_acquire);
+    if (scratch == nullptr) {
+        e = cudaGetSymbolAddress(&scratch, g_bb_static_scratch);
         if (e != cudaSuccess) return e;
-        g_bb_static_ptr[dev] = p;
+        g_bb_static_ptr[dev].store(scratch, std::memory_order_release);
     }
     int target = sm_count * 4 < kMaxFlatCtas ? sm_count * 4 : kMaxFlatCtas;
     FlatGrid g = make_flat_grid(total, target, 8192);
-    if (bb_ws_bytes(T, g.ctas) > kNoAllocBytes) return cudaErrorInvalidValue;
-    BbWs ws = bb_ws_carve(g_bb_static_ptr[dev], T, g.ctas);
+    // cannot happen for T <= kNoAllocMaxTensors (the caller checked): the array is sized for that many
+    // tensors and the largest grid
+    if (bb_ws_bytes(T, g.ctas) > kNoAllocBytes) return cudaErrorUnknown;
+    BbWs ws = bb_ws_carve(scratch, T, g.ctas);
     // the array still holds the previous call's counters: clear the part this call uses
-    e = cudaMemsetAsync(g_bb_static_ptr[dev], 0, bb_ws_bytes(T, g.ctas), stream);
+    e = cudaMemsetAsync(scratch, 0, bb_ws_bytes(T, g.ctas), stream);
     if (e != cudaSuccess) return e;
     for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
         launch_begin("k_bb_pass", stream);

@@ -237,6 +237,16 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
     });
 }
 
+// Two fp32 additions in one instruction (each rounded to nearest): (a0, a1) += (b0, b1).
+__device__ __forceinline__ void add2(float& a0, float& a1, float b0, float b1)
+{
+    unsigned long long a, b;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(b0), "f"(b1));
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(a) : "l"(b));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(a));
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(kThreads)
 k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* __restrict__ levels_k, int K,
@@ -289,10 +299,12 @@ k_unpack_sum(const uint32_t* const* __restrict__ packed_k, const float* const* _
                 // adds the levels of the four codes of this lane in word w (worker row r) to a[0..3]
                 auto add4 = [&](uint32_t w, const char* r, float* a) {
                     const uint32_t f = (w >> shift) << 2;  // byte offsets of the 4 codes
-                    a[0] = __fadd_rn(a[0], *reinterpret_cast<const float*>(r + (f & (kMask1 << 2))));
-                    a[1] = __fadd_rn(a[1], *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2))));
-                    a[2] = __fadd_rn(a[2], *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2))));
-                    a[3] = __fadd_rn(a[3], *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2))));
+                    const float l0 = *reinterpret_cast<const float*>(r + (f & (kMask1 << 2)));
+                    const float l1 = *reinterpret_cast<const float*>(r + ((f >> BITS) & (kMask1 << 2)));
+                    const float l2 = *reinterpret_cast<const float*>(r + ((f >> (2 * BITS)) & (kMask1 << 2)));
+                    const float l3 = *reinterpret_cast<const float*>(r + ((f >> (3 * BITS)) & (kMask1 << 2)));
+                    add2(a[0], a[1], l0, l1);  // same fp32 additions, two per instruction
+                    add2(a[2], a[3], l2, l3);
                 };
                 // two groups per warp and trip: sixteen word loads in flight per lane
                 for (int gl = warp; gl < ng; gl += 2 * kWarps) {

@@ -17,7 +17,7 @@
 // is found with one atomic counter per tensor.
 #include <math.h>
 
-#include <vector>
+#include <atomic>
 
 #include "ogq_common.cuh"
 #include "ogq_internal.h"
@@ -48,34 +48,14 @@ static_assert(kRound1Cells <= kCells, "round-1 cells exceed the budget");
 struct TState {
     int done, round, m, hi_e;
     unsigned kmin_inv, kmax, nonfinite, arrive;
-    unsigned expected, pad0;
+    unsigned expected;
+    int compact_only;  // the next pass only copies the keys inside the intervals: they fit one sort
     unsigned long long cursor[2];
     long long n;
     double stot;
     Interval iv[kMaxIv];
     ExactLv lv[kMaxLv];
-#ifdef OGQ_SOLVER_TIMING
-    long long tick[16];  // clock64() stamps of the last solver pass (debug builds only)
-#endif
 };
-
-#ifdef OGQ_SOLVER_TIMING
-#define OGQ_TICK(st, i) do { if (threadIdx.x == 0) (st)->tick[i] = clock64(); } while (0)
-// per-CTA wall-clock record of the round-1 and round-2 kernels: start, end, time in solver passes, passes
-__device__ unsigned long long g_dbg_cta[2][4096][8];
-__device__ __forceinline__ unsigned long long dbg_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define OGQ_CTA_BEGIN(k) unsigned long long dbg_t0 = dbg_now(), dbg_solver = 0, dbg_passes = 0, dbg_ph[4] = {0, 0, 0, 0}, dbg_last = dbg_t0; const int dbg_k = (k);
-// adds the time since the previous mark to phase i (0 setup, 1 streaming, 2 flush, 3 combine / arrive)
-#define OGQ_CTA_PHASE(i) do { const unsigned long long n_ = dbg_now(); dbg_ph[i] += n_ - dbg_last; dbg_last = n_; } while (0)
-#define OGQ_CTA_SOLVER(expr) do { unsigned long long a_ = dbg_now(); expr; dbg_solver += dbg_now() - a_; ++dbg_passes; } while (0)
-#define OGQ_CTA_END() do { if (threadIdx.x == 0 && blockIdx.x < 4096) { g_dbg_cta[dbg_k][blockIdx.x][0] = dbg_t0; g_dbg_cta[dbg_k][blockIdx.x][1] = dbg_now(); g_dbg_cta[dbg_k][blockIdx.x][2] = dbg_solver; g_dbg_cta[dbg_k][blockIdx.x][3] = dbg_passes; for (int q_ = 0; q_ < 4; ++q_) g_dbg_cta[dbg_k][blockIdx.x][4 + q_] = dbg_ph[q_]; } } while (0)
-#else
-#define OGQ_TICK(st, i) do { } while (0)
-#define OGQ_CTA_BEGIN(k)
-#define OGQ_CTA_PHASE(i) do { } while (0)
-#define OGQ_CTA_SOLVER(expr) do { expr; } while (0)
-#define OGQ_CTA_END() do { } while (0)
-#endif
 
 struct SelWs {
     TState* st;                  // [T]
@@ -488,6 +468,7 @@ struct Round2Ctx {  // per-CTA constants of round 2, kept in shared memory to sp
     uint32_t* dst;
     unsigned long long* cursor;
     uint32_t clear;  // 0x7fffffff when only magnitudes count
+    int nohist;      // copy the keys inside the intervals without counting them
 };
 
 // Phase B of round 2 for one warp: classifies `fill` parked values 32 at a time.  A free function
@@ -509,7 +490,7 @@ __device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx,
             int cell, sh;
             uint32_t low;
             in = classify(*tb, key, cell, low, sh);
-            if (in) hist_add(ctx->cnt, ctx->lo, ctx->hi, cell, low);
+            if (in && !ctx->nohist) hist_add(ctx->cnt, ctx->lo, ctx->hi, cell, low);
         }
         const uint32_t m2 = __ballot_sync(0xffffffffu, in);
         if (m2) {
@@ -590,7 +571,7 @@ struct Round2Warp {
 __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64_t pb, int64_t pe,
                                               bool magnitude_only, const Table& tb, uint32_t* cnt, uint32_t* lo,
                                               uint32_t* hi, uint32_t* stage, uint32_t* dst,
-                                              unsigned long long* cursor)
+                                              unsigned long long* cursor, bool nohist)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __shared__ Round2Ctx ctx;
@@ -599,6 +580,7 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
     if (threadIdx.x == 0) {
         ctx.cnt = cnt; ctx.lo = lo; ctx.hi = hi; ctx.dst = dst; ctx.cursor = cursor;
         ctx.clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
+        ctx.nohist = nohist ? 1 : 0;
     }
     if (lane == 0) fills[warp] = 0;
     __syncthreads();
@@ -667,13 +649,13 @@ template <bool FIRST, bool FROM_GRAD, bool COMPACT>
 __device__ __forceinline__ void stream_piece(const void* __restrict__ src, int64_t pb, int64_t pe,
                                              bool magnitude_only, const Table& tb, uint32_t* cnt,
                                              uint32_t* lo, uint32_t* hi, Stager& stg, uint32_t& kmin,
-                                             uint32_t& kmax, uint32_t& nonfinite)
+                                             uint32_t& kmax, uint32_t& nonfinite, bool nohist = false)
 {
     auto handle = [&](uint32_t key, uint32_t* kk, int& c) {
         int cell, sh;
         uint32_t low;
         if (classify(tb, key, cell, low, sh)) {
-            hist_add(cnt, lo, hi, cell, low);
+            if (!nohist) hist_add(cnt, lo, hi, cell, low);
             if (COMPACT) kk[c++] = key;
         }
     };
@@ -898,7 +880,6 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
         f_hi[threadIdx.x] = real ? S.niv[threadIdx.x].khi : 0u;
     }
     __syncthreads();
-    OGQ_TICK(st, 10);
     {
         const int lane = threadIdx.x & 31;
         constexpr int kCols = 8;
@@ -953,16 +934,13 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
             }
         }
     }
-    OGQ_TICK(st, 11);
     __syncthreads();
     const int c = S.n_keys < kSmallN ? S.n_keys : kSmallN;
     int P = 1;
     while (P < c) P <<= 1;
-    OGQ_TICK(st, 6);
     for (int i = c + threadIdx.x; i < kSmallN; i += kSelThreads) skeys[i] = 0xffffffffu;
     __syncthreads();
     block_bitonic_sort(skeys, P);
-    OGQ_TICK(st, 7);
     // pass 1: run starts and value sums of this thread's kPer consecutive sorted elements
     const int base = threadIdx.x * kPer;
     uint32_t k[kPer];
@@ -983,7 +961,14 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
     double sbase = ls, tsum;
     block_excl_scan(ubase, sbase, S.sc, S.ss, tu, tsum);
     if (threadIdx.x == 0) S.n_unique = (int)tu;
-    OGQ_TICK(st, 8);
+    // interval of each of this thread's keys, of the key before them and of the key after them
+    // (searched once; the passes below reuse them)
+    int jv[kPer];
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) jv[e] = (base + e < c) ? find_new_interval(S, k[e]) : -1;
+    const int jprev = (base > 0 && base <= c) ? find_new_interval(S, prev) : -2;
+    const uint32_t knext = (base + kPer < c) ? skeys[base + kPer] : 0u;
+    const int jnext = (base + kPer < c) ? find_new_interval(S, knext) : -3;
     // pass 2: first element of every interval
     {
         int nf = 0;
@@ -995,8 +980,8 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
                 const uint32_t pk = (e == 0) ? prev : k[e - 1];
                 const bool flag = (i == 0) || (k[e] != pk);
                 if (flag) {
-                    const int j = find_new_interval(S, k[e]);
-                    const int jp = (i == 0) ? -2 : find_new_interval(S, pk);
+                    const int j = jv[e];
+                    const int jp = (i == 0) ? -2 : ((e == 0) ? jprev : jv[e - 1]);
                     if (j >= 0 && j != jp) {
                         S.ivstart[j] = i;
                         S.ivpre[j] = run;
@@ -1019,7 +1004,7 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
             if (i < c) {
                 const uint32_t pk = (e == 0) ? prev : k[e - 1];
                 const bool flag = (i == 0) || (k[e] != pk);
-                const int j = find_new_interval(S, k[e]);
+                const int j = jv[e];
                 const double val = (double)sel_key_to_float(k[e]);
                 if (flag) {
                     const int u = (int)ubase + nf;
@@ -1030,8 +1015,8 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
                     }
                     ++nf;
                 }
-                const uint32_t nk = (i + 1 < c) ? ((e + 1 < kPer) ? k[e + 1] : skeys[i + 1]) : 0u;
-                const bool last_of_iv = (i + 1 >= c) || (find_new_interval(S, nk) != j);
+                const int jn = (i + 1 < c) ? ((e + 1 < kPer) ? jv[e + 1] : jnext) : -4;
+                const bool last_of_iv = (i + 1 >= c) || (jn != j);
                 if (last_of_iv && j >= 0) {
                     const int u = (int)ubase + nf - 1;
                     xcpre[u + 1 + j] = (uint32_t)(S.niv[j].cbefore + (long long)(i + 1 - S.ivstart[j]));
@@ -1061,12 +1046,12 @@ __device__ void sort_finish(TState* st, int t, int s, const uint32_t* buf, long 
         sel_init_slots(S.view);
         S.internal = (S.n_keys > kSmallN) ? 1 : 0;
     }
-    OGQ_TICK(st, 9);
     // one thread per level, one depth at a time (every cell is a single key now, so each solve is exact)
     for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
         __syncthreads();
-        const int q = threadIdx.x;
-        if (!S.internal && q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0 && !S.lv[q].exact) {
+        const int q = threadIdx.x >> 5;  // one warp per level, as in solver_round
+        if ((threadIdx.x & 31) == 0 && !S.internal && q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0 &&
+            !S.lv[q].exact) {
             if (!sel_orq_solve(S.view, S.lv[q - stride], S.lv[q + stride], S.lv[q])) S.internal = 1;
         }
     }
@@ -1214,7 +1199,6 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     uint8_t* slot_iv = smem + kOffSpre + kSlots * sizeof(double);
     const bool pb = scheme == OGQ_BINGRAD_PB;
     const int round = st->round;
-    OGQ_TICK(st, 0);
 
     __syncthreads();
     if ((int)threadIdx.x < st->m) S.iv[threadIdx.x] = st->iv[threadIdx.x];
@@ -1252,19 +1236,37 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         }
         __syncthreads();
         // raw (count, sum) of every cell: strided so that the global loads are coalesced and independent
-#pragma unroll 4
-        for (int slot = threadIdx.x; slot < nslots; slot += kSelThreads) {
-            const int jj = slot_iv[slot];
-            const int c = slot - S.view.slotbase[jj];
-            unsigned long long cn = 0;
-            double sm = 0.0;
-            if (c < S.iv[jj].ncell) {
-                cn = __ldcg(gcnt + S.iv[jj].cellbase + c);
-                const unsigned long long lsum = __ldcg(glsum + S.iv[jj].cellbase + c);
-                sm = sel_cell_sum(S.iv[jj].klo + ((uint32_t)c << S.iv[jj].sh), S.iv[jj].sh, cn, lsum);
+        // (all of a thread's loads are issued before the first is used: they come from L2)
+        constexpr int kPerThread = (kSlots + kSelThreads - 1) / kSelThreads;
+        uint32_t rc[kPerThread];
+        unsigned long long rl[kPerThread];
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u) {
+            const int slot = threadIdx.x + u * kSelThreads;
+            rc[u] = 0u;
+            rl[u] = 0ull;
+            if (slot < nslots) {
+                const int jj = slot_iv[slot];
+                const int c = slot - S.view.slotbase[jj];
+                if (c < S.iv[jj].ncell) {
+                    rc[u] = __ldcg(gcnt + S.iv[jj].cellbase + c);
+                    rl[u] = __ldcg(glsum + S.iv[jj].cellbase + c);
+                }
             }
-            cpre[slot] = (uint32_t)cn;
-            spre[slot] = sm;
+        }
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u) {
+            const int slot = threadIdx.x + u * kSelThreads;
+            if (slot < nslots) {
+                double sm = 0.0;
+                if (rc[u]) {
+                    const int jj = slot_iv[slot];
+                    const int c = slot - S.view.slotbase[jj];
+                    sm = sel_cell_sum(S.iv[jj].klo + ((uint32_t)c << S.iv[jj].sh), S.iv[jj].sh, rc[u], rl[u]);
+                }
+                cpre[slot] = rc[u];
+                spre[slot] = sm;
+            }
         }
         __syncthreads();
         // exclusive prefix: per-thread blocks, one block scan, in place
@@ -1306,7 +1308,6 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         S.view.stot = st->stot;
     }
     __syncthreads();
-    OGQ_TICK(st, 1);
 
     if (pb && !S.internal && S.view.stot > 0.0) {
         // bracket of the sign change of g, evaluated at the lower edge of every cell
@@ -1344,16 +1345,20 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
                 l.c_lt = e.c_lt; l.c_le = e.c_le; l.s_lt = e.s_lt; l.s_le = e.s_le;
             }
         }
+        // (one warp per level: the solves of one depth are long chains of dependent shared-memory
+        // reads and fp64 divisions, and lanes of one warp that take different branches would run
+        // one after the other)
+        static_assert(kSelWarps >= kMaxLv - 1, "one warp per interior level");
         for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
             __syncthreads();
-            const int q = threadIdx.x;
-            if (q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0 && !S.lv[q].exact) {
+            const int q = threadIdx.x >> 5;
+            if ((threadIdx.x & 31) == 0 && q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0 &&
+                !S.lv[q].exact) {
                 if (!sel_orq_solve(S.view, S.lv[q - stride], S.lv[q + stride], S.lv[q])) S.internal = 1;
             }
         }
     }
     __syncthreads();
-    OGQ_TICK(st, 2);
 
     if (threadIdx.x == 0) {
         int open = 0;
@@ -1425,32 +1430,33 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
             }
         }
     }
-    OGQ_TICK(st, 3);
     __syncthreads();
 
     if (S.done) {
         if (threadIdx.x == 0) { st->done = 1; __threadfence(); }
-        OGQ_TICK(st, 5);
         return true;
     }
     if (!pb && round >= 2 && S.cand <= kSmallN && round_buf != nullptr) {
         const long long src_cnt = (long long)__ldcg(&st->cursor[round & 1]);
         if (src_cnt <= kSortScanMax) {
-            OGQ_TICK(st, 4);
             sort_finish(st, t, s, round_buf, src_cnt, levels, status, smem, S);
-            OGQ_TICK(st, 5);
             return true;
         }
     }
-    // prepare the next round: clear the cells it will use, publish the new intervals
+    // prepare the next round: clear the cells it will use, publish the new intervals.  When the
+    // elements inside the new intervals already fit one sort (ORQ), the next pass only copies them
+    // and its last CTA sorts and finishes the tensor (finish_sorted): no cells, no further solver pass.
+    const bool compact_only = !pb && S.cand <= kSmallN;
     const int ncells_next = S.niv[S.nm - 1].cellbase + S.niv[S.nm - 1].ncell;
-    for (int i = threadIdx.x; i < ncells_next; i += kSelThreads) {
-        gcnt[i] = 0u;
-        glsum[i] = 0ull;
-    }
+    if (!compact_only)
+        for (int i = threadIdx.x; i < ncells_next; i += kSelThreads) {
+            gcnt[i] = 0u;
+            glsum[i] = 0ull;
+        }
     if ((int)threadIdx.x < S.nm) st->iv[threadIdx.x] = S.niv[threadIdx.x];
     if (threadIdx.x == 0) {
         st->m = S.nm;
+        st->compact_only = compact_only ? 1 : 0;
         st->round = round + 1;
         st->arrive = 0;
         const int next = round + 1;
@@ -1467,8 +1473,35 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     }
     __threadfence();
     __syncthreads();
-    OGQ_TICK(st, 5);
     return false;
+}
+
+// Finishes a tensor whose last pass only copied the keys inside its intervals (TState::compact_only):
+// the solver state the previous pass left in global memory is loaded back, then the copied keys are
+// sorted and every open level is solved on single-key cells.  Called by every thread of the CTA that
+// arrived last for the tensor.
+__device__ void finish_sorted(TState* st, int t, int s, const uint32_t* copied, float* __restrict__ levels,
+                              int32_t* __restrict__ status, unsigned char* smem, SolverShared& S, int cursor_idx)
+{
+    __syncthreads();
+    const int m = __ldcg(&st->m);
+    if ((int)threadIdx.x < m) S.niv[threadIdx.x] = st->iv[threadIdx.x];
+    if ((int)threadIdx.x < s) {
+        const ExactLv& e = st->lv[threadIdx.x];
+        LvInfo& l = S.lv[threadIdx.x];
+        l.exact = e.exact; l.key = e.key; l.val = (double)sel_key_to_float(e.key);
+        l.c_lt = e.c_lt; l.c_le = e.c_le; l.s_lt = e.s_lt; l.s_le = e.s_le;
+        l.sa = l.sb = 0; l.vlo = l.vhi = l.val;
+    }
+    if (threadIdx.x == 0) {
+        S.nm = m;
+        S.view.n = st->n;
+        S.view.stot = st->stot;
+        S.internal = 0;
+    }
+    __syncthreads();
+    const long long src_cnt = (long long)__ldcg(&st->cursor[cursor_idx]);
+    sort_finish(st, t, s, copied, src_cnt, levels, status, smem, S);
 }
 
 // ---------------------------------------------------------------------------
@@ -1631,10 +1664,11 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
         const int round = st->round;
         const uint32_t* src = A.ws.buf[(round - 1) & 1];  // 16-byte aligned base; indices are absolute
         const int64_t cnt = (int64_t)__ldcg(&st->cursor[(round - 1) & 1]);
+        const bool copy_only = st->compact_only != 0;
         __syncthreads();
         if (threadIdx.x == 0) table_from_intervals(tb, st->iv, st->m);
         __syncthreads();
-        zero_hist(hist, tb.ncells);
+        if (!copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
         Stager stg;
         stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
@@ -1643,9 +1677,15 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
         stg.fill = 0;
         uint32_t kmin = 0, kmax = 0, nf = 0;
         stream_piece<false, false, true>(src, tbeg, tbeg + cnt, false, tb, hist, hist + kCells, hist + 2 * kCells,
-                                         stg, kmin, kmax, nf);
+                                         stg, kmin, kmax, nf, copy_only);
         stg.flush();
         __syncthreads();
+        if (copy_only) {
+            __threadfence();
+            __syncthreads();
+            finish_sorted(st, t, A.s, A.ws.buf[round & 1] + tbeg, A.levels, A.status, smem, S, round & 1);
+            return;
+        }
         flush_hist(hist, tb.ncells, gcnt, glsum);
         __threadfence();
         __syncthreads();
@@ -1671,15 +1711,10 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
     const int nl = pb ? 2 : A.s;
 
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
-    OGQ_CTA_BEGIN(0)
 
-    // Round 1 over one piece [pb_, pe_) of tensor t.  `alone`: the piece is the whole tensor and
-    // this CTA runs all of its rounds.  Returns true when the tensor is finished.
-    auto do_round1 = [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_, bool alone) -> bool {
-        const int64_t n = tend - tbeg;
-        TState* st = A.ws.st + t;
-        // anchor of the fine window: largest binade among strided samples, plus two (every CTA of the
-        // tensor samples the same elements and so arrives at the same window)
+    // Anchor of the fine window of tensor [tbeg, tbeg + n): largest binade among strided samples, plus
+    // two (every CTA of the tensor samples the same elements and so arrives at the same window).
+    auto window_anchor = [&](int64_t tbeg, int64_t n) -> int {
         int hi_e;
         {
             const int64_t idx = tbeg + (int64_t)threadIdx.x * n / kSelThreads;
@@ -1693,6 +1728,16 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
             if (hi_e < kSelW) hi_e = kSelW;
             if (hi_e > 255) hi_e = 255;  // binade 255 (Inf / NaN) always stays outside the fine window
         }
+        return hi_e;
+    };
+
+    // Round 1 over one piece [pb_, pe_) of tensor t: histogram, min / max, arrival.  `alone`: the piece
+    // is the whole tensor.  Returns true when this CTA is the last one of the tensor to arrive; that
+    // CTA then runs r1_solve.
+    auto r1_stream = [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_, bool alone) -> bool {
+        const int64_t n = tend - tbeg;
+        TState* st = A.ws.st + t;
+        const int hi_e = window_anchor(tbeg, n);
         const int lo_e = hi_e - kSelW;
         const int ncells = pb ? kRound1Mag : kRound1Cells;
         uint32_t* gcnt = A.ws.gcnt + (size_t)t * kCells;
@@ -1701,11 +1746,9 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         uint32_t nf = 0u;
         zero_hist(hist, ncells);
         __syncthreads();
-        OGQ_CTA_PHASE(0);
         if (pb) stream_round1<true>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf);
         else stream_round1<false>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf);
         __syncthreads();
-        OGQ_CTA_PHASE(1);
         // The low sums of the window's cells are 32 bits wide without a carry: exact as long as no such
         // cell took more than 2^16 values.  Otherwise (heavily repeated values) the piece is redone in
         // parts of kR1MaxPiece elements, flushed one by one.
@@ -1731,7 +1774,6 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         } else {
             flush_hist(hist, ncells, gcnt, glsum);
         }
-        OGQ_CTA_PHASE(2);
         // min / max / non-finite: one atomic per warp
         {
             const uint32_t kmin = __reduce_min_sync(0xffffffffu, float_to_key(vmin));  // +Inf / -Inf when the
@@ -1752,11 +1794,18 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
                 sh_last = (prev == (unsigned)(c1 - c0));
             }
             __syncthreads();
-            OGQ_CTA_PHASE(3);
             if (!sh_last) return false;
             __threadfence();
         }
-        // last CTA of this tensor: set up the state and run the first solver pass
+        return true;
+    };
+
+    // Last CTA of tensor t: sets up the state and runs the first solver pass.  Returns true when the
+    // tensor is finished.
+    auto r1_solve = [&](int t, int64_t tbeg, int64_t tend, bool alone) -> bool {
+        const int64_t n = tend - tbeg;
+        TState* st = A.ws.st + t;
+        const int hi_e = window_anchor(tbeg, n);
         __syncthreads();
         if (threadIdx.x == 0) {
             st->n = n;
@@ -1783,9 +1832,9 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         __syncthreads();
         if (sh_last & (OGQ_ST_NONFINITE | OGQ_ST_CONSTANT)) return true;
         bool done;
-        OGQ_CTA_SOLVER(done = solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells,
+        done = solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells,
                                            A.scheme, A.s, A.levels, A.status, A.ws.nitems, A.ws.items, nullptr,
-                                           !alone, smem, S));
+                                           !alone, smem, S);
         return done;
     };
 
@@ -1802,42 +1851,36 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         } else if (n <= kSmallN) {
             small_tensor(A.grad, tbeg, (int)n, t, A.scheme, A.s, A.levels, A.status, A.ws.st + t, smem);
         } else if (n <= kMidN) {
-            // all rounds on this CTA: round 1 and 2 read the tensor (it stays in L2), later rounds the copied keys
-            if (do_round1(t, tbeg, tend, tbeg, tend, true)) return;
-            TState* st = A.ws.st + t;
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                table_from_intervals(tb, st->iv, st->m);
-                tb.lo_e = st->hi_e - kSelW;
-            }
-            __syncthreads();
-            build_prefilter(tb, pb);
-            zero_hist(hist, tb.ncells);
-            __syncthreads();
-            stream_round2(A.grad, tbeg, tend, pb, tb, hist, hist + kCells, hist + 2 * kCells,
-                          reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
-                          A.ws.buf[0] + tbeg, &st->cursor[0]);
-            __syncthreads();
-            flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
-            __threadfence();
-            __syncthreads();
-            if (solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                             A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, false, smem, S))
-                return;
-            finish_alone(A, t, smem, tb, S);
+            // round 1 and its solver pass on this CTA; the tensor's CTA of the round-2 kernel goes on from there
+            r1_stream(t, tbeg, tend, tbeg, tend, true);
+            r1_solve(t, tbeg, tend, true);
         }
         }();
-        OGQ_CTA_END();
         return;
     }
 
     const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
     const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+    // A CTA first streams all of its pieces and only then runs the solver passes of the tensors it
+    // finished, so that a solver pass never holds up the arrival of another tensor's piece.
+    constexpr int kDefer = 8;
+    int dt[kDefer];
+    int nd = 0;
     for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
         if (tend - tbeg <= kMidN) return;
-        do_round1(t, tbeg, tend, pb_, pe_, false);
+        if (!r1_stream(t, tbeg, tend, pb_, pe_, false)) return;
+        if (nd < kDefer) {
+#pragma unroll
+            for (int u = 0; u < kDefer; ++u)
+                if (u == nd) dt[u] = t;
+            ++nd;
+        } else {
+            r1_solve(t, tbeg, tend, false);
+        }
     });
-    OGQ_CTA_END();
+#pragma unroll
+    for (int u = 0; u < kDefer; ++u)
+        if (u < nd) r1_solve(dt[u], __ldg(A.off + dt[u]), __ldg(A.off + dt[u] + 1), false);
 }
 
 __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArgs A)
@@ -1847,45 +1890,93 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
     __shared__ SolverShared S;
     __shared__ int sh_last;
     const bool pb = A.scheme == OGQ_BINGRAD_PB;
-    const int64_t lo = (int64_t)blockIdx.x * A.chunk;
-    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
-    OGQ_CTA_BEGIN(1)
 
+    // Second pass over the piece [pb_, pe_) of tensor t: copies the values inside the tensor's
+    // intervals (and counts them on the finer cells unless they already fit one sort).
+    auto r2_stream = [&](int t, int64_t tbeg, int64_t pb_, int64_t pe_, bool& copy_only) {
+        TState* st = A.ws.st + t;
+        __syncthreads();
+        table_from_intervals_cta(tb, st->iv, __ldcg(&st->m));
+        __syncthreads();
+        build_prefilter(tb, pb);
+        copy_only = __ldcg(&st->compact_only) != 0;
+        if (!copy_only) zero_hist(hist, tb.ncells);
+        __syncthreads();
+        stream_round2(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells,
+                      reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
+                      A.ws.buf[0] + tbeg, &st->cursor[0], copy_only);
+        __syncthreads();
+        if (!copy_only) flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+        __threadfence();
+        __syncthreads();
+    };
+
+    if ((int)blockIdx.x < A.T) {
+        // the first T CTAs, one per tensor, take the mid-size tensors from where their CTA of the
+        // round-1 kernel left them to the end (the tensor stays in L2, later rounds read copied keys)
+        const int t = blockIdx.x;
+        const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
+        const int64_t n = tend - tbeg;
+        TState* st = A.ws.st + t;
+        if (n <= kSmallN || n > kMidN || __ldcg(&st->done)) return;
+        bool copy_only;
+        r2_stream(t, tbeg, tbeg, tend, copy_only);
+        if (copy_only) {
+            finish_sorted(st, t, A.s, A.ws.buf[0] + tbeg, A.levels, A.status, smem, S, 0);
+            return;
+        }
+        if (solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
+                         A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, false, smem, S))
+            return;
+        finish_alone(A, t, smem, tb, S);
+        return;
+    }
+
+    const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
+    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+    // as in round 1, the solver passes of the tensors this CTA finished wait until all of its pieces
+    // have been streamed
+    constexpr int kDefer = 8;
+    int dt[kDefer];
+    int nd = 0;
+    auto finish = [&](int t) {
+        TState* st = A.ws.st + t;
+        const int64_t tbeg = __ldg(A.off + t);
+        if (__ldcg(&st->compact_only) != 0) {
+            finish_sorted(st, t, A.s, A.ws.buf[0] + tbeg, A.levels, A.status, smem, S, 0);
+            return;
+        }
+        solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
+                     A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, true, smem, S);
+    };
     for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
         const int64_t n = tend - tbeg;
         if (n <= kMidN) return;
         TState* st = A.ws.st + t;
         if (__ldcg(&st->done)) return;
-        __syncthreads();
-        table_from_intervals_cta(tb, st->iv, __ldcg(&st->m));
-        __syncthreads();
-        build_prefilter(tb, pb);
-        zero_hist(hist, tb.ncells);
-        __syncthreads();
-        OGQ_CTA_PHASE(0);
-        stream_round2(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells,
-                      reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
-                      A.ws.buf[0] + tbeg, &st->cursor[0]);
-        __syncthreads();
-        OGQ_CTA_PHASE(1);
-        flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
-        __threadfence();
-        __syncthreads();
-        OGQ_CTA_PHASE(2);
+        bool copy_only;
+        r2_stream(t, tbeg, pb_, pe_, copy_only);
         const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
         if (threadIdx.x == 0) {
             const unsigned prev = atomicAdd(&st->arrive, 1u);
             sh_last = (prev == (unsigned)(c1 - c0));
         }
         __syncthreads();
-        OGQ_CTA_PHASE(3);
         if (!sh_last) return;
         __threadfence();
-        OGQ_CTA_SOLVER(solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme,
-                                    A.s, A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, true, smem, S));
+        if (nd < kDefer) {
+#pragma unroll
+            for (int u = 0; u < kDefer; ++u)
+                if (u == nd) dt[u] = t;
+            ++nd;
+        } else {
+            finish(t);
+        }
     });
-    OGQ_CTA_END();
+#pragma unroll
+    for (int u = 0; u < kDefer; ++u)
+        if (u < nd) finish(dt[u]);
 }
 
 __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArgs A)
@@ -1911,8 +2002,9 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
         if (pe_ > cnt) pe_ = cnt;
         __syncthreads();
         if (threadIdx.x == 0) table_from_intervals(tb, st->iv, __ldcg(&st->m));
+        const bool copy_only = __ldcg(&st->compact_only) != 0;
         __syncthreads();
-        zero_hist(hist, tb.ncells);
+        if (!copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
         Stager stg;
         stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
@@ -1921,10 +2013,10 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
         stg.fill = 0;
         uint32_t kmin = 0, kmax = 0, nf = 0;
         stream_piece<false, false, true>(A.ws.buf[0], tbeg + pb_, tbeg + pe_, false, tb, hist, hist + kCells,
-                                         hist + 2 * kCells, stg, kmin, kmax, nf);
+                                         hist + 2 * kCells, stg, kmin, kmax, nf, copy_only);
         stg.flush();
         __syncthreads();
-        flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+        if (!copy_only) flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         __threadfence();
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -1934,42 +2026,35 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
         __syncthreads();
         if (!sh_last) continue;
         __threadfence();
+        if (copy_only) {
+            finish_sorted(st, t, A.s, A.ws.buf[1] + tbeg, A.levels, A.status, smem, S, 1);
+            continue;
+        }
         if (!solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
                           A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[1] + tbeg, false, smem, S))
             finish_alone(A, t, smem, tb, S);
     }
 }
 
-#ifdef OGQ_SOLVER_TIMING
-extern "C" int ogq_debug_dump_ctas(unsigned long long* h_out /*[2][4096][8]*/)
-{
-    return cudaMemcpyFromSymbol(h_out, g_dbg_cta, sizeof(unsigned long long) * 2 * 4096 * 8) == cudaSuccess ? 0 : -1;
-}
-extern "C" int ogq_debug_dump_ticks(const void* d_ws, int T, long long* h_out /*[T][16]*/, int* h_round, long long* h_n)
-{
-    std::vector<TState> h(T);
-    if (cudaMemcpy(h.data(), d_ws, sizeof(TState) * (size_t)T, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
-    for (int t = 0; t < T; ++t) {
-        for (int i = 0; i < 16; ++i) h_out[t * 16 + i] = h[t].tick[i];
-        h_round[t] = h[t].round;
-        h_n[t] = h[t].n;
-    }
-    return 0;
-}
-#endif
-
 cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int T, int64_t total, int scheme,
                                  int s, float* d_levels, int32_t* d_status, void* d_ws, size_t /*ws_bytes*/,
                                  int sm_count, cudaStream_t stream)
 {
     {
-        cudaError_t e;
-        e = cudaFuncSetAttribute(k_sel_round1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        // the kernels need more dynamic shared memory than the default limit: raised once per device
+        static std::atomic<bool> attr_set[64];
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_sel_round2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
+            e = cudaFuncSetAttribute(k_sel_round1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            if (e != cudaSuccess) return e;
+            e = cudaFuncSetAttribute(k_sel_round2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            if (e != cudaSuccess) return e;
+            e = cudaFuncSetAttribute(k_sel_round3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
+        }
     }
     // Flat streaming CTAs: one wave (kSelResident per SM).  Each CTA pays a set-up, a flush of its
     // cells and an arrival per tensor piece, so larger chunks stream more of the time; a second wave
@@ -1988,7 +2073,7 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     k_sel_round1<<<g.ctas + T, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     launch_begin("k_sel_round2", stream);
-    k_sel_round2<<<g.ctas, kSelThreads, kSmemBytes, stream>>>(A);
+    k_sel_round2<<<g.ctas + T, kSelThreads, kSmemBytes, stream>>>(A);
     launch_end(stream);
     launch_begin("k_sel_round3", stream);
     k_sel_round3<<<kSelResident * sm_count, kSelThreads, kSmemBytes, stream>>>(A);

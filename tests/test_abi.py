@@ -51,3 +51,17 @@ def test_workspace_bytes_is_monotone_and_positive():
     b = ogq.ogq_workspace_bytes(161, 25557032, 17)
     assert 0 < a <= b
     assert ogq.ogq_workspace_bytes(-1, 5, 3) == 0
+
+
+def test_selection_solvers_refuse_buckets_of_2_to_the_32_elements():
+    """The ORQ and BinGrad-pb solvers count in 32-bit cells: the header gives the limit and the call
+    returns OGQ_ERR_UNSUPPORTED before it touches the device (no GPU needed for this check)."""
+    big = 1 << 32
+    dummy = 256  # never dereferenced: the size check comes first
+    with pytest.raises(ogq.OgqError) as e:
+        ogq.ogq_levels_orq(dummy, dummy, 1, big, 9, dummy, dummy, dummy, 1 << 40, stream=0)
+    assert e.value.code == 2
+    with pytest.raises(ogq.OgqError) as e:
+        ogq.ogq_levels_bingrad(dummy, dummy, 1, big, ogq.OGQ_BINGRAD_PB, 0, dummy, dummy, dummy, dummy, 1 << 40,
+                               stream=0)
+    assert e.value.code == 2

@@ -23,12 +23,29 @@ if torch.cuda.is_available():
 ORACLE_MAX = 5_000_000  # tensors up to this size get the element-by-element oracle
 
 
-def check_orq_levels_by_condition(v, lv):
+class SortedView:
+    """The tensor sorted once (fp32 comparisons are exact) with fp64 prefix sums, so that the checks
+    below cost a few binary searches per level whatever the tensor's size."""
+
+    def __init__(self, v):
+        self.sv = np.sort(v)
+        self.cs = np.zeros(v.size + 1, np.float64)
+        np.cumsum(self.sv, dtype=np.float64, out=self.cs[1:])
+
+    def segment(self, L, R):
+        """(count, sum) of {L <= v <= R} and the index range in the sorted array."""
+        i0 = int(np.searchsorted(self.sv, L, side="left"))
+        i1 = int(np.searchsorted(self.sv, R, side="right"))
+        return i0, i1, self.cs[i1] - self.cs[i0]
+
+
+def check_orq_levels_by_condition(v, lv, view=None):
     """Each level is a data value and satisfies, against the two levels it was solved from,
-    count{b <= v <= R} >= T >= count{b < v <= R} with T = sum_{L<=v<=R}(v - L)/(R - L).
-    Works on the fp32 array directly (comparisons of fp32 values are exact), sums in fp64."""
+    count{b <= v <= R} >= T >= count{b < v <= R} with T = sum_{L<=v<=R}(v - L)/(R - L)
+    (discrete form of the simplified optimal condition, applied in the order of Algorithm 1)."""
+    view = view if view is not None else SortedView(v)
     s = lv.size
-    assert lv[0] == v.min() and lv[-1] == v.max()
+    assert lv[0] == view.sv[0] and lv[-1] == view.sv[-1]
 
     def rec(l, r):
         if r - l < 2:
@@ -36,11 +53,13 @@ def check_orq_levels_by_condition(v, lv):
         m = (l + r) // 2
         L, R, b = lv[l], lv[r], lv[m]
         if R > L:
-            seg = v[(v >= L) & (v <= R)]
-            T = (np.sum(seg, dtype=np.float64) - float(L) * seg.size) / (float(R) - float(L))
-            ge, gt = int(np.count_nonzero(seg >= b)), int(np.count_nonzero(seg > b))
+            i0, i1, ssum = view.segment(L, R)
+            cnt = i1 - i0
+            T = (ssum - float(L) * cnt) / (float(R) - float(L))
+            ge = i1 - int(np.searchsorted(view.sv, b, side="left"))
+            gt = i1 - int(np.searchsorted(view.sv, b, side="right"))
             assert ge > gt, "level is not a data value"
-            slack = 1e-9 * seg.size
+            slack = 1e-9 * cnt
             assert ge >= T - slack and gt <= T + slack, (l, r, ge, gt, T)
         else:
             assert b == L
@@ -48,6 +67,22 @@ def check_orq_levels_by_condition(v, lv):
         rec(m, r)
 
     rec(0, s - 1)
+
+
+def check_pb_level_by_condition(v, b1):
+    """BinGrad-pb: g(b) = b n - sum_{|v| >= b} |v| is increasing in b and the level sits at its sign
+    change (Eq. (bingrad-pb optimal condition) on magnitudes), so g is <= 0 one fp32 step below the
+    level and >= 0 one step above it, up to the rounding of the fp64 sums."""
+    a = np.abs(v)
+    n = a.size
+    b1 = np.float32(b1)
+    lo, hi = np.nextafter(b1, np.float32(-np.inf)), np.nextafter(b1, np.float32(np.inf))
+
+    def g(b):
+        return float(b) * n - float(np.sum(a[a >= b], dtype=np.float64))
+
+    tol = 1e-9 * n * float(b1) + 1e-300
+    assert b1 >= 0 and g(lo) <= tol and g(hi) >= -tol, (b1, g(lo), g(hi))
 
 
 def levels_close(got, want):
@@ -61,9 +96,23 @@ def worker_variants(db, K):
     return [g0 if k == 0 else (torch.roll(g0, 1001 * k) * (1.0 + 0.03 * k)).contiguous() for k in range(K)]
 
 
-def run_bucket(bucket, orq_levels, with_bingrad_b):
+def run_bucket(bucket, orq_levels, with_bingrad_b, with_bingrad_pb=True):
     db = DeviceBucket(bucket.values, bucket.offsets)
     sizes = np.diff(bucket.offsets)
+    if with_bingrad_pb:
+        lv, _, st = db.levels_bingrad(ogq.OGQ_BINGRAD_PB, 0)
+        assert not np.any(st & (ogq.OGQ_ST_INTERNAL | ogq.OGQ_ST_ITER_CAP | ogq.OGQ_ST_NONFINITE))
+        for t in range(db.T):
+            v = bucket.tensor(t)
+            assert lv[t][0] == -lv[t][1]
+            if sizes[t] <= ORACLE_MAX:
+                want, _ = oracle.levels_bingrad_pb(v)
+                assert levels_close(lv[t], want), (t, lv[t], want)
+            else:
+                check_pb_level_by_condition(v, lv[t][1])
+        got, _ = db.quantize_pack(ogq.OGQ_BINGRAD_PB, 2, lv, None, 3, 2)
+        want, _ = oracle.bucket_quantize_pack(bucket.values, bucket.offsets, oracle.PB, 2, lv, None, 3, 2)
+        assert np.array_equal(got, want)
     for s in orq_levels:
         lv, st = db.levels_orq(s)
         assert not np.any(st & (ogq.OGQ_ST_INTERNAL | ogq.OGQ_ST_ITER_CAP | ogq.OGQ_ST_NONFINITE))
@@ -141,11 +190,70 @@ def check_unpack_sum(db, s, K, full):
                 assert np.all(np.abs(got[a + e0 : a + e0 + m].astype(np.float64) - want) <= tol), (t, e0)
 
 
+def check_independent_workers(make_bucket, scheme, s, K):
+    """K workers with independent data seeds: each worker's bucket is generated, quantized on the GPU
+    and dropped again, only its levels and packed words are kept; then one unpack + sum over the K
+    buffers.  Every worker's packed words and the whole dequantized sum are compared with the oracle."""
+    b0 = make_bucket(0)
+    db = DeviceBucket(b0.values, b0.offsets)
+    bits = ogq.ogq_bits_for_levels(s)
+    h_po = ogq.ogq_packed_layout(db.h_off, bits)
+    po = torch.from_numpy(h_po).to(db.dev)
+    lvs, pks = [], []
+    for k in range(K):
+        b = b0 if k == 0 else make_bucket(k)
+        assert np.array_equal(b.offsets, b0.offsets)
+        grad = db.grad if k == 0 else torch.from_numpy(b.values).to(db.dev)
+        st = torch.zeros(db.T, dtype=torch.int32, device=db.dev)
+        pk = torch.zeros(int(h_po[-1]), dtype=torch.int32, device=db.dev)
+        if scheme == ogq.OGQ_ORQ:
+            lv = torch.zeros((db.T, s), device=db.dev)
+            ogq.ogq_levels_orq(grad, db.off, db.T, db.N, s, lv, st, db.ws, db.ws_bytes)
+            ogq.ogq_quantize_pack(grad, db.off, db.T, db.N, scheme, s, lv, None, 5, k, po, pk)
+            th = None
+        else:
+            lv = torch.zeros((db.T, 2), device=db.dev)
+            th = torch.zeros(db.T, device=db.dev)
+            ogq.ogq_levels_bingrad(grad, db.off, db.T, db.N, scheme, 0, lv, th, st, db.ws, db.ws_bytes)
+            ogq.ogq_quantize_pack(grad, db.off, db.T, db.N, scheme, 2, lv, th, 5, k, po, pk)
+        torch.cuda.synchronize()
+        assert not np.any(st.cpu().numpy() & (ogq.OGQ_ST_INTERNAL | ogq.OGQ_ST_ITER_CAP | ogq.OGQ_ST_NONFINITE))
+        h_lv = lv.cpu().numpy()
+        h_th = th.cpu().numpy() if th is not None else None
+        want, _ = oracle.bucket_quantize_pack(b.values, b.offsets, scheme, s, h_lv, h_th, 5, k)
+        assert np.array_equal(pk.cpu().numpy().view(np.uint32), want), k
+        if scheme == ogq.OGQ_BINGRAD_B:
+            w_lv, w_th, _ = oracle.bucket_levels_bingrad(b.values, b.offsets, oracle.B, 0)
+            for t in range(db.T):
+                assert levels_close(h_lv[t], w_lv[t]), (k, t)
+        lvs.append(lv)
+        pks.append(pk)
+        del grad, b
+    out = torch.empty(db.N, device=db.dev)
+    ogq.ogq_unpack_sum(ogq.device_pointer_array(pks), ogq.device_pointer_array(lvs), K, db.off, po, db.T, db.N, s,
+                       1.0 / K, out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    want = oracle.bucket_unpack_sum([p.cpu().numpy().view(np.uint32) for p in pks], [l.cpu().numpy() for l in lvs],
+                                    db.h_off, s, 1.0 / K)
+    for t in range(db.T):
+        a, e = int(db.h_off[t]), int(db.h_off[t + 1])
+        if e > a:
+            tol = 1e-5 * float(np.max(np.abs(want[a:e])))
+            assert np.all(np.abs(got[a:e].astype(np.float64) - want[a:e]) <= tol), t
+
+
 def test_resnet50_bucket_full_size():
     b = wl.resnet50_bucket(0)
     assert b.num_tensors == 161 and b.total == 25557032
-    db = run_bucket(b, orq_levels=(3, 9), with_bingrad_b=False)
+    db = run_bucket(b, orq_levels=(3, 9), with_bingrad_b=True)
     check_unpack_sum(db, 9, 8, full=True)
+    check_unpack_sum(db, 3, 8, full=True)
+
+
+@pytest.mark.parametrize("s", [3, 9])
+def test_resnet50_eight_independent_workers(s):
+    check_independent_workers(wl.resnet50_bucket, ogq.OGQ_ORQ, s, 8)
 
 
 def test_vgg19_bucket_full_size():
@@ -155,24 +263,37 @@ def test_vgg19_bucket_full_size():
     check_unpack_sum(db, 9, 8, full=False)
 
 
+def test_vgg19_bingrad_b_eight_independent_workers():
+    check_independent_workers(wl.vgg19_bucket, ogq.OGQ_BINGRAD_B, 2, 8)
+
+
 @pytest.mark.parametrize("log2n", [20, 24, 26, 28])
 def test_flat_sweep_tensor(log2n):
     b = wl.sweep_tensor(log2n)
     db = DeviceBucket(b.values, b.offsets)
-    for s in ((3, 5, 9, 17) if log2n <= 24 else (9,)):
+    view = SortedView(b.values) if b.total > ORACLE_MAX else None
+    for s in (3, 5, 9, 17):
         lv, st = db.levels_orq(s)
         assert st[0] == 0
         if b.total <= ORACLE_MAX:
             want, _ = oracle.levels_orq(b.values, s)
             assert np.array_equal(lv[0], want)
         else:
-            check_orq_levels_by_condition(b.values, lv[0])
+            check_orq_levels_by_condition(b.values, lv[0], view)
         got, _ = db.quantize_pack(ogq.OGQ_ORQ, s, lv, None, 7, 1)
         want, _ = oracle.bucket_quantize_pack(b.values, b.offsets, oracle.ORQ, s, lv, None, 7, 1)
         assert np.array_equal(got, want)
-    lv, th, _ = db.levels_bingrad(ogq.OGQ_BINGRAD_B, 0)
-    w_lv, w_th, _ = oracle.bucket_levels_bingrad(b.values, b.offsets, oracle.B, 0)
-    assert levels_close(lv[0], w_lv[0])
+    del view
+    # BinGrad-b: levels, 1-bit codes, and the unpack of K = 1 worker (the dequantized gradient itself)
+    lv, th, st = db.levels_bingrad(ogq.OGQ_BINGRAD_B, 0)
+    w_lv, w_th, w_st = oracle.bucket_levels_bingrad(b.values, b.offsets, oracle.B, 0)
+    assert st[0] == w_st[0] and levels_close(lv[0], w_lv[0])
+    assert abs(float(th[0]) - float(w_th[0])) <= 1e-5 * float(np.abs(w_lv[0]).max())
+    got, _ = db.quantize_pack(ogq.OGQ_BINGRAD_B, 2, lv, th, 0, 0)
+    want, _ = oracle.bucket_quantize_pack(b.values, b.offsets, oracle.B, 2, lv, th, 0, 0)
+    assert np.array_equal(got, want)
+    out = db.unpack_sum([got], [lv], 2, 1.0)
+    assert np.array_equal(out, oracle.bucket_unpack_sum([want], [lv], b.offsets, 2, 1.0))
 
 
 def test_flat_tensor_with_crowded_cells():

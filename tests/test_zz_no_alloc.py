@@ -5,7 +5,8 @@ fires in the middle of a step, or a process whose memory pool another framework 
 ogq_levels_bingrad_b_noalloc, which keeps the solver's counters in an array built into the library.
 This file checks that it gives the same levels, thresholds and status words as ogq_levels_bingrad
 (same tolerance as the other level tests: 1e-5 of the tensor's largest level), on two calls in a row
-that reuse the built-in array with different buckets, and that it refuses more tensors than it holds.
+that reuse the built-in array with different buckets, at the largest tensor count it accepts, that it
+leaves the amount of device memory in use unchanged, and that it refuses more tensors than it holds.
 It is collected last on purpose, and it also passes when run alone in a fresh process.
 """
 import numpy as np
@@ -62,6 +63,42 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
     # second call reuses the built-in array: fewer tensors, other data, Lloyd updates
     b = wl.config2()
     _assert_same(_run_both(b.values, b.offsets, 3))
+
+
+def test_noalloc_at_its_capacity_then_a_small_call():
+    """T = 1024 puts the per-tensor counters at the far end of the built-in array; the small call that
+    follows must not be disturbed by what the large one left there."""
+    r = np.random.Generator(np.random.PCG64(31))
+    sizes = [int(x) for x in r.integers(0, 3000, 1024)]
+    sizes[5] = sizes[700] = sizes[1023] = 0
+    sizes[17] = 300001
+    parts = [wl.laplace(r, n, 10.0 ** r.uniform(-5, -2)) if n else np.zeros(0, np.float32) for n in sizes]
+    _assert_same(_run_both(np.concatenate(parts), wl.offsets_from_sizes(sizes), 2))
+    vals, h_off = _bucket(22)
+    _assert_same(_run_both(vals, h_off, 1))
+
+
+def test_noalloc_call_leaves_device_memory_in_use_unchanged():
+    """What the entry point is for: the free device memory the driver reports is the same before and
+    after calls (outputs and inputs are allocated by the test beforehand; torch's caching allocator
+    is not asked for anything in between)."""
+    dev = torch.device("cuda:0")
+    vals, h_off = _bucket(23)
+    T, N = h_off.size - 1, int(h_off[-1])
+    grad = torch.from_numpy(vals).to(dev)
+    off = torch.from_numpy(h_off).to(dev)
+    lv = torch.zeros((T, 2), device=dev)
+    th = torch.zeros(T, device=dev)
+    st = torch.zeros(T, dtype=torch.int32, device=dev)
+    ogq.ogq_levels_bingrad_b_noalloc(grad, off, T, N, 0, lv, th, st)  # first call: address lookup
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info(dev)
+    reserved0 = torch.cuda.memory_reserved(dev)
+    for _ in range(3):
+        ogq.ogq_levels_bingrad_b_noalloc(grad, off, T, N, 2, lv, th, st)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info(dev)
+    assert free1 == free0 and torch.cuda.memory_reserved(dev) == reserved0
 
 
 def test_noalloc_rejects_more_tensors_than_it_holds():
