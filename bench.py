@@ -9,13 +9,18 @@ levels + quantize + pack (4 bytes x elements x K per step) over the step time.
     python bench.py --gpus 1 --steps 10 --warmup 3
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
     python bench.py --impl reference        # times the CPU oracle on a bounded sample
+    python bench.py --workload resnet50 --bucket-len 512   # fixed-length bucket mode
 
-Prints one JSON line (rank 0).
+Prints one JSON line (rank 0).  Besides the headline (K workers on K streams) the line carries the
+same stage with all workers on one stream (`single_stream`) and, for the default configuration,
+short runs of the other headline workloads and schemes (`secondary`).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import multiprocessing
 import os
 import statistics
 import subprocess
@@ -124,32 +129,64 @@ class ClockSampler:
 # --------------------------------------------------------------------------- CPU oracle arm
 
 
-def oracle_sample(workload: str, scheme_name: str, seconds: float = 15.0):
-    """Times the CPU oracle (levels + quantize + pack) on a bounded sample of worker 0's bucket:
-    a prefix of its largest tensor sized for about `seconds` of single-threaded work."""
+def _oracle_task(task):
+    """levels + quantize + pack of one tensor by the oracle (runs in a worker process)."""
+    v, scheme, s, lloyd = task
     import oracle
 
-    scheme, s, lloyd = SCHEMES[scheme_name]
-    b = make_bucket(workload, 0)
-    sizes = np.diff(b.offsets)
-    t_big = int(np.argmax(sizes))
-    big = b.tensor(t_big)
+    off = np.array([0, v.size], np.int64)
+    if scheme == 2:
+        lv, _ = oracle.bucket_levels_orq(v, off, s)
+        oracle.bucket_quantize_pack(v, off, oracle.ORQ, s, lv, None, 1, 0)
+    else:
+        lv, th, _ = oracle.bucket_levels_bingrad(v, off, scheme, lloyd)
+        oracle.bucket_quantize_pack(v, off, scheme, 2, lv, th, 1, 0)
+    return v.size
 
-    def run(v):
+
+class OraclePool:
+    """The machine's host cores as oracle workers (spawned, so that no CUDA state is inherited)."""
+
+    def __init__(self, cores=None):
+        self.cores = cores or os.cpu_count() or 1
+        self.pool = multiprocessing.get_context("spawn").Pool(self.cores)
+        self.pool.map(_oracle_task, [(np.zeros(64, np.float32), 2, 3, 0)] * self.cores)  # load the library
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
+
+    def sample(self, workload: str, scheme_name: str, seconds: float):
+        """A bounded sample of worker 0's bucket, sized for about `seconds` on all cores: whole tensors
+        where they are small enough, the first kCap elements of the larger ones (the sort-based oracle
+        grows faster than linearly), largest pieces dropped first when the estimate is still too long."""
+        kCap = 1 << 22
+        scheme, s, lloyd = SCHEMES[scheme_name]
+        b = make_bucket(workload, 0)
+        sizes = np.diff(b.offsets)
+        probe = b.tensor(int(np.argmax(sizes)))[: 1 << 18]
         t0 = time.perf_counter()
-        off = np.array([0, v.size], np.int64)
-        if scheme == 2:
-            lv, _ = oracle.bucket_levels_orq(v, off, s)
-            oracle.bucket_quantize_pack(v, off, oracle.ORQ, s, lv, None, 1, 0)
+        _oracle_task((probe, scheme, s, lloyd))
+        unit = (time.perf_counter() - t0) / (probe.size * np.log2(probe.size))  # seconds per n log2 n
+        pieces = [b.tensor(t)[:kCap] for t in range(b.num_tensors) if sizes[t] > 0]
+        pieces.sort(key=lambda v: v.size)
+        cost = lambda v: unit * v.size * max(1.0, np.log2(max(v.size, 2)))
+        while len(pieces) > self.cores and sum(cost(v) for v in pieces) / self.cores > seconds:
+            pieces.pop()
+        used = int(sum(v.size for v in pieces))
+        capped = int(sum(1 for v in pieces if v.size == kCap))
+        if used == b.total:
+            what = f"whole bucket of worker 0 ({b.num_tensors} tensors, {b.total} elements)"
         else:
-            lv, th, _ = oracle.bucket_levels_bingrad(v, off, scheme, lloyd)
-            oracle.bucket_quantize_pack(v, off, scheme, 2, lv, th, 1, 0)
-        return time.perf_counter() - t0
+            what = (f"{len(pieces)} of the {b.num_tensors} tensors of worker 0's bucket, smallest first, {capped} of them "
+                    f"cut to their first {kCap} elements ({used} of {b.total} elements)")
+        tasks = [(v, scheme, s, lloyd) for v in reversed(pieces)]
+        return tasks, used, what
 
-    probe = min(big.size, 1 << 17)
-    rate = probe / max(run(big[:probe]), 1e-9)  # elements per second
-    m = int(min(big.size, max(probe, rate * seconds)))
-    return big[:m], run, f"first {m} elements of the largest tensor ({sizes[t_big]} elements) of worker 0"
+    def run(self, tasks) -> float:
+        t0 = time.perf_counter()
+        self.pool.map(_oracle_task, tasks, chunksize=1)
+        return time.perf_counter() - t0
 
 
 def run_reference(args):
@@ -158,20 +195,22 @@ def run_reference(args):
         return
     steps, warmup = max(1, args.steps), max(0, args.warmup)
     budget = 150.0 / (steps + warmup)
-    v, run, what = oracle_sample(args.workload, args.scheme, seconds=min(15.0, budget))
+    pool = OraclePool()
+    tasks, used, what = pool.sample(args.workload, args.scheme, seconds=min(12.0, budget))
     for _ in range(warmup):
-        run(v)
+        pool.run(tasks)
     t0 = time.perf_counter()
     for _ in range(steps):
-        run(v)
+        pool.run(tasks)
     dt = (time.perf_counter() - t0) / steps
-    value = 4.0 * v.size / dt / 1e9
+    pool.close()
+    value = 4.0 * used / dt / 1e9
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "scheme": args.scheme, "sample": what},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": pool.cores, "kind": "oracle", "sample": what},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -181,15 +220,136 @@ def run_reference(args):
 # --------------------------------------------------------------------------- CUDA arm
 
 
+def kernel_sources_hash() -> str:
+    """sha256 over the kernel sources and the header: the key of the stored DRAM-traffic figures."""
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2002_11082_b200", "csrc")
+    for name in sorted(os.listdir(csrc)) + ["../../include/ogq.h"]:
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()
+
+
+def stored_traffic(kernel: str, scheme: str):
+    """DRAM bytes per element of `kernel` from the committed ncu summary, or None when the kernels have
+    changed since it was taken (the file records the hash of the sources it was measured on)."""
+    path = os.path.join(ROOT, "profiles", "dram_bytes_per_element.json")
+    try:
+        rec = json.load(open(path))
+        if rec.get("sources_sha256") != kernel_sources_hash():
+            return None
+        return rec["entries"].get(f"{kernel}|{scheme}")
+    except Exception:
+        return None
+
+
+class Setup:
+    """One workload x scheme resident in HBM: K workers' buckets, outputs, scratch, streams."""
+
+    def __init__(self, torch, ogq, dev, workload, scheme_name, K, seed, rank, bucket_len=0, share=None):
+        from paper_2002_11082_b200.sharding import worker_ids
+
+        self.torch, self.ogq, self.dev = torch, ogq, dev
+        self.workload, self.scheme_name, self.K, self.seed = workload, scheme_name, K, seed
+        self.scheme, self.s, self.lloyd = SCHEMES[scheme_name]
+        self.bits = ogq.ogq_bits_for_levels(self.s)
+        self.bucket_len = bucket_len
+        self.clip_c = 0.0
+        if share is not None and share.workload == workload:
+            self.host, self.grads = share.host, share.grads
+        else:
+            self.host = [make_bucket(workload, w) for w in worker_ids(rank, K)]
+            self.grads = [torch.from_numpy(h.values).to(dev) for h in self.host]
+        self.N = self.host[0].total
+        if bucket_len:
+            nb = (self.N + bucket_len - 1) // bucket_len
+            self.h_off = np.minimum(np.arange(nb + 1, dtype=np.int64) * bucket_len, self.N)
+        else:
+            self.h_off = self.host[0].offsets
+        self.T = self.h_off.size - 1
+        T, s = self.T, self.s
+        self.off = torch.from_numpy(self.h_off).to(dev)
+        self.h_po = ogq.ogq_packed_layout(self.h_off, self.bits)
+        self.po = torch.from_numpy(self.h_po).to(dev)
+        self.levels = [torch.zeros((T, s), device=dev) for _ in range(K)]
+        self.thresh = [torch.zeros((T,), device=dev) for _ in range(K)]
+        self.status = [torch.zeros((T,), dtype=torch.int32, device=dev) for _ in range(K)]
+        self.packed = [torch.zeros((int(self.h_po[-1]),), dtype=torch.int32, device=dev) for _ in range(K)]
+        self.ws_bytes = 256 if bucket_len else ogq.ogq_workspace_bytes(T, self.N, max(s, 3))
+        self.wss = [torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev) for _ in range(K)]
+        self.side = [torch.cuda.Stream(device=dev) for _ in range(K)]
+        self.out = torch.empty(self.N, device=dev)
+        self.pk_ptrs = ogq.device_pointer_array(self.packed)
+        self.lv_ptrs = ogq.device_pointer_array(self.levels)
+        self.grad_bytes = 4.0 * self.N * K
+        self.alg_lqp = (8.0 + self.bits / 8.0) * self.N * K
+
+    def lqp(self, k, stream=None, slot=None):
+        """levels + quantize + pack of worker k (scratch slot = the stream's own)."""
+        ogq, s = self.ogq, self.s
+        ws = self.wss[k if slot is None else slot]
+        if self.bucket_len:
+            ogq.ogq_bucket_encode(self.grads[k], self.N, self.bucket_len, self.scheme, s, 0, self.clip_c, self.seed, k,
+                                  self.levels[k], self.thresh[k], self.status[k], self.packed[k], stream)
+        elif self.scheme == ogq.OGQ_ORQ:
+            ogq.ogq_levels_orq(self.grads[k], self.off, self.T, self.N, s, self.levels[k], self.status[k], ws,
+                               self.ws_bytes, stream)
+            ogq.ogq_quantize_pack(self.grads[k], self.off, self.T, self.N, self.scheme, s, self.levels[k], None,
+                                  self.seed, k, self.po, self.packed[k], stream)
+        else:
+            ogq.ogq_levels_bingrad(self.grads[k], self.off, self.T, self.N, self.scheme, self.lloyd, self.levels[k],
+                                   self.thresh[k], self.status[k], ws, self.ws_bytes, stream)
+            ogq.ogq_quantize_pack(self.grads[k], self.off, self.T, self.N, self.scheme, 2, self.levels[k],
+                                  self.thresh[k], self.seed, k, self.po, self.packed[k], stream)
+
+    def unpack(self):
+        self.ogq.ogq_unpack_sum(self.pk_ptrs, self.lv_ptrs, self.K, self.off, self.po, self.T, self.N, self.s,
+                                1.0 / self.K, self.out)
+
+    def lqp_all(self, n_streams, before=None):
+        """levels + quantize + pack of all K workers, worker k on stream k mod n_streams;
+        `before(k)` runs on worker k's stream first."""
+        torch, K = self.torch, self.K
+        if n_streams <= 1:
+            for k in range(K):
+                if before is not None:
+                    before(k)
+                self.lqp(k, None, 0)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        for st in self.side[:n_streams]:
+            st.wait_event(fork)
+        for k in range(K):
+            st = self.side[k % n_streams]
+            with torch.cuda.stream(st):
+                if before is not None:
+                    before(k)
+                self.lqp(k, st, k % n_streams)
+        for st in self.side[:n_streams]:
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
+
+    def check_status(self):
+        bad = [int(st.bitwise_and(16 | 8).count_nonzero().item()) for st in self.status]
+        if any(bad):
+            raise SystemExit(f"solver reported unresolved tensors: {bad}")
+
+
 def run_ours(args):
-    import torch
-
-    import paper_2002_11082_b200 as ogq
-    from paper_2002_11082_b200.sharding import aggregate_throughput, max_over_ranks, worker_ids
-
+    # the oracle's worker processes are started before the first CUDA call
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    pool = OraclePool() if (rank == 0 and world == 1 and not args.no_cpu) else None
+
+    import torch
+
+    import paper_2002_11082_b200 as ogq
+    from paper_2002_11082_b200.sharding import aggregate_throughput, max_over_ranks
+
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -201,72 +361,10 @@ def run_ours(args):
         dist_mod.init_process_group("nccl", device_id=dev)
         dist = dist_mod
 
-    scheme, s, lloyd = SCHEMES[args.scheme]
     K = args.workers
-    bits = ogq.ogq_bits_for_levels(s)
-
-    # ---- inputs: K workers' buckets, generated on the host and made resident in HBM
-    host = [make_bucket(args.workload, w) for w in worker_ids(rank, K)]
-    h_off = host[0].offsets
-    T, N = host[0].num_tensors, host[0].total
-    off = torch.from_numpy(h_off).to(dev)
-    h_po = ogq.ogq_packed_layout(h_off, bits)
-    po = torch.from_numpy(h_po).to(dev)
-    grads = [torch.from_numpy(h.values).to(dev) for h in host]
-    levels = [torch.zeros((T, s), device=dev) for _ in range(K)]
-    thresh = [torch.zeros((T,), device=dev) for _ in range(K)]
-    status = [torch.zeros((T,), dtype=torch.int32, device=dev) for _ in range(K)]
-    packed = [torch.zeros((int(h_po[-1]),), dtype=torch.int32, device=dev) for _ in range(K)]
-    ws_bytes = ogq.ogq_workspace_bytes(T, N, max(s, 3))
-    # workers alternate between `args.streams` CUDA streams, each with its own scratch, so that the
-    # short single-CTA solver tails of one worker overlap the streaming kernels of the next
     n_streams = max(1, min(args.streams, K))
-    wss = [torch.empty(ws_bytes, dtype=torch.uint8, device=dev) for _ in range(n_streams)]
-    side = [torch.cuda.Stream(device=dev) for _ in range(n_streams)] if n_streams > 1 else []
-    out = torch.empty(N, device=dev)
-    pk_ptrs = ogq.device_pointer_array(packed)
-    lv_ptrs = ogq.device_pointer_array(levels)
-
-    def lqp(k, stream=None):
-        ws = wss[k % n_streams]
-        if scheme == ogq.OGQ_ORQ:
-            ogq.ogq_levels_orq(grads[k], off, T, N, s, levels[k], status[k], ws, ws_bytes, stream)
-            ogq.ogq_quantize_pack(grads[k], off, T, N, scheme, s, levels[k], None, args.seed, k, po, packed[k], stream)
-        else:
-            ogq.ogq_levels_bingrad(grads[k], off, T, N, scheme, lloyd, levels[k], thresh[k], status[k], ws, ws_bytes,
-                                   stream)
-            ogq.ogq_quantize_pack(grads[k], off, T, N, scheme, 2, levels[k], thresh[k], args.seed, k, po, packed[k],
-                                  stream)
-
-    def unpack():
-        ogq.ogq_unpack_sum(pk_ptrs, lv_ptrs, K, off, po, T, N, s, 1.0 / K, out)
-
-    def lqp_all(before=None):
-        """levels + quantize + pack of all K workers; `before(k)` runs on worker k's stream first."""
-        if n_streams == 1:
-            for k in range(K):
-                if before is not None:
-                    before(k)
-                lqp(k)
-            return
-        main = torch.cuda.current_stream()
-        fork = torch.cuda.Event()
-        fork.record(main)
-        for st in side:
-            st.wait_event(fork)
-        for k in range(K):
-            with torch.cuda.stream(side[k % n_streams]):
-                if before is not None:
-                    before(k)
-                lqp(k, side[k % n_streams])
-        for st in side:
-            join = torch.cuda.Event()
-            join.record(st)
-            main.wait_event(join)
-
-    def step():
-        lqp_all()
-        unpack()
+    peak, peak_src = measured_peaks()
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     def barrier():
         torch.cuda.synchronize()
@@ -274,12 +372,9 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    # L2 hygiene: the large buckets cycle through far more than the 126 MB L2 per step; for the small
-    # workloads a buffer larger than L2 is overwritten before every timed step, outside the timed events
-    need_flush = 4 * N * K <= 2 * 126e6
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
-
-    def timed(fn, reps):
+    def timed(fn, reps, need_flush):
+        """Device time of `reps` calls of fn (CUDA events on the current stream, max over ranks).
+        Small workloads: a buffer larger than L2 is overwritten before every call, outside the events."""
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         if not need_flush:
@@ -300,35 +395,48 @@ def run_ours(args):
         barrier()
         return max_over_ranks(total, dist, dev)
 
+    S = Setup(torch, ogq, dev, args.workload, args.scheme, K, args.seed, rank, args.bucket_len)
+    N, T, bits, s = S.N, S.T, S.bits, S.s
+    # L2 hygiene: the large buckets cycle through far more than the 126 MB L2 per step
+    need_flush = 4 * N * K <= 2 * 126e6
+
+    def step():
+        S.lqp_all(n_streams)
+        S.unpack()
+
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     for _ in range(warmup):
         step()
     torch.cuda.synchronize()
-    bad = [int(st.bitwise_and(16 | 8).count_nonzero().item()) for st in status]
-    if any(bad):
-        raise SystemExit(f"solver reported unresolved tensors: {bad}")
+    S.check_status()
 
     # ---- the timed region: exactly `steps` steps
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     launches0 = ogq.ogq_launch_count()
-    ms_total = timed(step, steps)
+    ms_total = timed(step, steps, need_flush)
     launches = ogq.ogq_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     ms_step = ms_total / steps
-    grad_bytes = 4.0 * N * K  # fp32 gradient consumed per step and rank
-    value = aggregate_throughput(grad_bytes, ms_step, world)
+    value = aggregate_throughput(S.grad_bytes, ms_step, world)
+
+    def stage_block(setup, streams, reps, flush):
+        ms = timed(lambda: setup.lqp_all(streams), reps, flush) / reps
+        gbs = setup.alg_lqp / (ms * 1e-3) / 1e9
+        return {"streams": streams, "ms": ms, "grad_gbs": setup.grad_bytes / (ms * 1e-3) / 1e9,
+                "alg_bytes_per_elem": 8.0 + setup.bits / 8.0, "frac_of_hbm_peak": gbs / peak,
+                "frac_of_nominal_8tbs": gbs / 8000.0}
 
     # ---- per-stage and per-kernel times (separate instrumented passes, not part of `value`)
-    ms_lqp = timed(lqp_all, steps) / steps
-    ms_unp = timed(unpack, steps) / steps
+    st_multi = stage_block(S, n_streams, steps, need_flush)
+    st_single = stage_block(S, 1, steps, need_flush)
+    ms_unp = timed(S.unpack, steps, need_flush) / steps
     ogq.ogq_profile_enable(True)  # per-kernel times: one stream, so that no two kernels overlap
     torch.cuda.synchronize()
     for _ in range(steps):
-        for k in range(K):
-            lqp(k)
-        unpack()
+        S.lqp_all(1)
+        S.unpack()
     torch.cuda.synchronize()
     recs = ogq.ogq_profile_collect()
     ogq.ogq_profile_enable(False)
@@ -339,9 +447,8 @@ def run_ours(args):
     alg_bytes = {  # algorithmic bytes of one launch, per the accounting in the design notes
         "k_sel_round1": 4.0 * N, "k_sel_round2": 4.0 * N, "k_sel_round3": 0.0, "k_bb_pass": 4.0 * N,
         "k_quantize_pack_random": (4.0 + bits / 8.0) * N, "k_quantize_pack_threshold": (4.0 + 1 / 8.0) * N,
-        "k_unpack_sum": (K * bits / 8.0 + 4.0) * N,
+        "k_unpack_sum": (K * bits / 8.0 + 4.0) * N, "k_bucket_encode": (4.0 + bits / 8.0) * N,
     }
-    peak, peak_src = measured_peaks()
     kernels = {}
     total_ms = max(sum(v[0] for v in per_kernel.values()), 1e-12)
     for name, (tot, cnt) in per_kernel.items():
@@ -349,61 +456,72 @@ def run_ours(args):
         gbs = alg_bytes.get(name, 0.0) / (avg * 1e-3) / 1e9 if avg > 0 else 0.0
         kernels[name] = {"launches_per_step": cnt / steps, "avg_ms": avg, "share": tot / total_ms, "alg_gbs": gbs}
     dom = max(per_kernel, key=lambda k: per_kernel[k][0])
-    # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from one ncu
-    # capture of the current kernels on a 2^26-element tensor with s = 9; traffic grows in proportion to
-    # the elements streamed, so a full launch is this figure times N.  Other schemes: not captured.
-    ncu_dram_bytes_per_element = {"k_sel_round1": 4.461, "k_sel_round2": 4.232, "k_quantize_pack_random": 4.397}
-    traffic = None
-    if args.scheme == "orq9" and dom in ncu_dram_bytes_per_element:
-        traffic = ncu_dram_bytes_per_element[dom] * N
+    per_elem = stored_traffic(dom, args.scheme if not args.bucket_len else f"{args.scheme}_d{args.bucket_len}")
     roofline = {
         "bound": "hbm", "kernel": dom, "achieved": kernels[dom]["alg_gbs"], "peak": peak, "unit": "GB/s",
-        "frac": kernels[dom]["alg_gbs"] / peak, "traffic": traffic, "peak_source": peak_src,
-        "alg_bytes_per_launch": alg_bytes.get(dom, 0.0),
+        "frac": kernels[dom]["alg_gbs"] / peak, "traffic": per_elem * N if per_elem is not None else None,
+        "peak_source": peak_src, "alg_bytes_per_launch": alg_bytes.get(dom, 0.0),
     }
 
     # ---- end to end through the C ABI with host buffers (H2D of every worker's bucket, D2H of the result)
     e2e = None
     if not args.no_e2e:
-        pinned = [torch.from_numpy(h.values).pin_memory() for h in host]
+        pinned = [torch.from_numpy(h.values).pin_memory() for h in S.host]
         h_out = torch.empty(N, dtype=torch.float32).pin_memory()
 
         def e2e_step():
-            lqp_all(before=lambda k: grads[k].copy_(pinned[k], non_blocking=True))
-            unpack()
-            h_out.copy_(out, non_blocking=True)
+            S.lqp_all(n_streams, before=lambda k: S.grads[k].copy_(pinned[k], non_blocking=True))
+            S.unpack()
+            h_out.copy_(S.out, non_blocking=True)
 
         e2e_steps = min(steps, 5)
         e2e_step()
-        ms_e2e = timed(e2e_step, e2e_steps) / e2e_steps
-        e2e = {"value": aggregate_throughput(grad_bytes, ms_e2e, world), "unit": UNIT,
+        ms_e2e = timed(e2e_step, e2e_steps, need_flush) / e2e_steps
+        e2e = {"value": aggregate_throughput(S.grad_bytes, ms_e2e, world), "unit": UNIT,
                "h2d_bytes_per_step": int(4 * N * K), "d2h_bytes_per_step": int(4 * N),
                "ms_per_step": ms_e2e, "steps": e2e_steps}
+        del pinned, h_out
 
-    # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only)
+    # ---- the other headline workloads and schemes, short runs (default configuration only)
+    secondary = None
+    if world == 1 and not args.no_secondary and args.workload == "vgg19" and args.scheme == "orq9" and not args.bucket_len:
+        secondary = {}
+        for wk, sch, blen in (("vgg19", "bingrad_b", 0), ("resnet50", "orq9", 0), ("resnet50", "orq3", 0),
+                              ("resnet50", "bingrad_b", 0), ("resnet50", "orq9", 512)):
+            X = Setup(torch, ogq, dev, wk, sch, K, args.seed, rank, blen, share=S)
+            flush = 4 * X.N * K <= 2 * 126e6
+            for _ in range(3):
+                X.lqp_all(n_streams)
+            torch.cuda.synchronize()
+            X.check_status()
+            key = f"{wk}_{sch}" + (f"_d{blen}" if blen else "")
+            secondary[key] = {"streams_K": stage_block(X, n_streams, 5, flush), "single_stream": stage_block(X, 1, 5, flush)}
+            del X
+            torch.cuda.empty_cache()
+
+    # ---- CPU oracle on a bounded sample, on all host cores (rank 0, single GPU runs only)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu:
-        v, run, what = oracle_sample(args.workload, args.scheme, seconds=args.cpu_seconds)
-        dt = run(v)
-        cpu = {"value": 4.0 * v.size / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what,
+    if pool is not None:
+        tasks, used, what = pool.sample(args.workload, args.scheme, seconds=args.cpu_seconds)
+        dt = pool.run(tasks)
+        cpu = {"value": 4.0 * used / dt / 1e9, "unit": UNIT, "cores": pool.cores, "kind": "oracle", "sample": what,
                "seconds": dt}
+        pool.close()
 
     if rank == 0:
-        alg_lqp = (8.0 + bits / 8.0) * N * K
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "scheme": args.scheme, "levels": s, "bits": bits,
                        "workers_per_gpu": K, "tensors": T, "elements": N, "streams": n_streams,
+                       "bucket_len": args.bucket_len or None,
                        "l2": "256 MB written between timed steps (flush)" if need_flush else "inputs larger than L2 (no flush)"},
             "stages": {
-                "levels_quantize_pack": {"ms": ms_lqp, "grad_gbs": grad_bytes / (ms_lqp * 1e-3) / 1e9,
-                                         "alg_bytes_per_elem": 8.0 + bits / 8.0,
-                                         "frac_of_hbm_peak": alg_lqp / (ms_lqp * 1e-3) / 1e9 / peak,
-                                         "frac_of_nominal_8tbs": alg_lqp / (ms_lqp * 1e-3) / 1e9 / 8000.0},
+                "levels_quantize_pack": st_multi,
                 "unpack_sum": {"ms": ms_unp, "alg_gbs": (K * bits / 8.0 + 4.0) * N / (ms_unp * 1e-3) / 1e9},
             },
+            "single_stream": st_single, "secondary": secondary,
             "kernels": kernels, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
         }
@@ -423,9 +541,12 @@ def main():
     ap.add_argument("--workers", type=int, default=8)
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--streams", type=int, default=8)
-    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true")
+    ap.add_argument("--bucket-len", type=int, default=0,
+                    help="fixed-length bucket mode: quantize buckets of this many elements (ogq_bucket_encode)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

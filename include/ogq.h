@@ -173,6 +173,70 @@ ogq_status ogq_unpack_sum(const uint32_t *const *d_packed_k, const float *const 
                           int s, float scale, float *d_out, ogq_stream_t stream);
 
 /*
+ * Gradient clipping (Section "Experiments", paragraph after the list of methods):
+ * clip(v) = sign(v) min(|v|, c sigma), sigma^2 the variance of the gradient being quantized
+ * (here: of each tensor, about its mean, over all its elements), c = 2.5 in the ImageNet runs,
+ * 1.7 or 2.5 in the clipping-factor table.
+ *   ogq_clip_threshold: d_tau[t] = fp32(c * sigma_t) from one streaming read; d_status[t] gets
+ *     OGQ_ST_EMPTY or OGQ_ST_NONFINITE (then d_tau[t] = 0), else 0.  Scratch as for
+ *     ogq_levels_bingrad (ogq_workspace_bytes).
+ *   ogq_levels_orq_clipped / ogq_levels_bingrad_clipped: the level solvers on the clipped
+ *     gradient; the clamp to [-d_tau[t], d_tau[t]] is applied as the values are read, the clipped
+ *     gradient is never written out.  ORQ's end levels become the clipped extremes.  A non-finite
+ *     value is clipped like any other, so it is ogq_clip_threshold that reports it.
+ *   ogq_quantize_pack_clipped: ogq_quantize_pack with the same clamp applied first, so that the
+ *     codes are exactly those of the clipped gradient (plain ogq_quantize_pack with the clipped
+ *     levels decodes to the same values but may pick another of several equal levels for a value
+ *     beyond +-tau).
+ */
+ogq_status ogq_clip_threshold(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems,
+                              float c, float *d_tau, int32_t *d_status, void *d_ws, size_t ws_bytes,
+                              ogq_stream_t stream);
+ogq_status ogq_levels_orq_clipped(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems,
+                                  int s, const float *d_tau, float *d_levels, int32_t *d_status,
+                                  void *d_ws, size_t ws_bytes, ogq_stream_t stream);
+ogq_status ogq_levels_bingrad_clipped(const float *d_grad, const int64_t *d_off, int T,
+                                      int64_t total_elems, int variant, int lloyd_iters,
+                                      const float *d_tau, float *d_levels, float *d_thresh,
+                                      int32_t *d_status, void *d_ws, size_t ws_bytes,
+                                      ogq_stream_t stream);
+ogq_status ogq_quantize_pack_clipped(const float *d_grad, const int64_t *d_off, int T,
+                                     int64_t total_elems, ogq_scheme scheme, int s,
+                                     const float *d_levels, const float *d_thresh, const float *d_tau,
+                                     uint64_t seed, uint32_t stream_id, const int64_t *d_packed_off,
+                                     uint32_t *d_packed, ogq_stream_t stream);
+
+/*
+ * Fixed-length bucket mode (Section "Experiments", first paragraph: "bucket-based quantization
+ * ... evenly divides the whole gradient into buckets of the same length d and quantizes each
+ * bucket independently"; d = 2048 on CIFAR, 512 on ImageNet, 128 ... 32768 in the bucket-size
+ * table).  One call does levels + quantize + pack for every bucket of d_grad[0 .. total_elems):
+ * bucket j is elements [j d, min((j+1) d, total_elems)), nb = ceil(total_elems / d) buckets.
+ * Each bucket is read from HBM once, sorted in shared memory, solved and packed by one CTA.
+ * The results are those of ogq_levels_* followed by ogq_quantize_pack on a bucket of nb tensors
+ * with offsets j d: same level definitions, Philox tensor index = j, and the packed layout of
+ * ogq_packed_layout for those offsets (bucket j starts at word j * d * bits / 32;
+ * ogq_bucket_packed_words gives the total).  ogq_unpack_sum decodes it with the same offsets.
+ *   d      multiple of 128, 128 <= d <= 32768 (else OGQ_ERR_UNSUPPORTED)
+ *   scheme OGQ_ORQ (s in {3, 5, 9, 17}), OGQ_BINGRAD_B or OGQ_BINGRAD_PB (s = 2)
+ *   iters  OGQ_ORQ: refinement sweeps after Algorithm 1 (0 = the paper's greedy levels).  One
+ *          sweep re-solves every interior level, in ascending order, from its two current
+ *          neighbours, b_k = Q*(b_{k-1}, b_{k+1}); sweeps stop early when one changes nothing
+ *          (the paper's conclusion names the greedy algorithm as open to improvement; each
+ *          sweep cannot increase the expected quantization error).
+ *          OGQ_BINGRAD_B: Lloyd updates, as lloyd_iters of ogq_levels_bingrad.  PB: ignored.
+ *   clip_c 0: no clipping.  > 0: every bucket is first clipped to +-clip_c times its own standard
+ *          deviation (see ogq_clip_threshold; ImageNet setting of the paper: d = 512, c = 2.5).
+ * Outputs: d_levels [nb][s], d_thresh [nb] (B only, may be NULL otherwise), d_status [nb],
+ * d_packed.  No scratch memory is needed.
+ */
+int64_t ogq_bucket_packed_words(int64_t total_elems, int d, int bits);
+ogq_status ogq_bucket_encode(const float *d_grad, int64_t total_elems, int d, ogq_scheme scheme, int s,
+                             int iters, float clip_c, uint64_t seed, uint32_t stream_id, float *d_levels,
+                             float *d_thresh, int32_t *d_status, uint32_t *d_packed,
+                             ogq_stream_t stream);
+
+/*
  * Measurement helpers (no counterpart in the paper; they do not touch the data path).
  * ogq_launch_count: number of kernels this library has launched in this process so far.
  * ogq_profile_enable(1): from now on every kernel launch of the library is bracketed by two CUDA

@@ -27,6 +27,12 @@ from .binding import (  # noqa: F401
     ogq_levels_orq,
     ogq_quantize_pack,
     ogq_unpack_sum,
+    ogq_clip_threshold,
+    ogq_levels_orq_clipped,
+    ogq_levels_bingrad_clipped,
+    ogq_quantize_pack_clipped,
+    ogq_bucket_packed_words,
+    ogq_bucket_encode,
     ogq_launch_count,
     ogq_profile_enable,
     ogq_profile_collect,

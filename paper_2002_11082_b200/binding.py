@@ -59,6 +59,20 @@ def lib() -> ctypes.CDLL:
         L.ogq_quantize_pack.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, ctypes.c_uint64, ctypes.c_uint32, vp, vp, vp]
         L.ogq_unpack_sum.restype = i32
         L.ogq_unpack_sum.argtypes = [vp, vp, i32, vp, vp, i32, i64, i32, ctypes.c_float, vp, vp]
+        L.ogq_bucket_packed_words.restype = i64
+        L.ogq_bucket_packed_words.argtypes = [i64, i32, i32]
+        L.ogq_bucket_encode.restype = i32
+        L.ogq_bucket_encode.argtypes = [vp, i64, i32, i32, i32, i32, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint32,
+                                        vp, vp, vp, vp, vp]
+        L.ogq_clip_threshold.restype = i32
+        L.ogq_clip_threshold.argtypes = [vp, vp, i32, i64, ctypes.c_float, vp, vp, vp, sz, vp]
+        L.ogq_levels_orq_clipped.restype = i32
+        L.ogq_levels_orq_clipped.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, sz, vp]
+        L.ogq_quantize_pack_clipped.restype = i32
+        L.ogq_quantize_pack_clipped.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, ctypes.c_uint64, ctypes.c_uint32,
+                                                vp, vp, vp]
+        L.ogq_levels_bingrad_clipped.restype = i32
+        L.ogq_levels_bingrad_clipped.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.ogq_launch_count.restype = ctypes.c_ulonglong
         L.ogq_launch_count.argtypes = []
         L.ogq_profile_enable.restype = i32
@@ -162,6 +176,59 @@ def ogq_unpack_sum(d_packed_k, d_levels_k, K: int, d_off, d_packed_off, T: int, 
         lib().ogq_unpack_sum(_ptr(d_packed_k), _ptr(d_levels_k), int(K), _ptr(d_off), _ptr(d_packed_off),
                              int(T), int(total_elems), int(s), float(scale), _ptr(d_out), _stream(stream)),
         "ogq_unpack_sum",
+    )
+
+
+def ogq_bucket_packed_words(total_elems: int, d: int, bits: int) -> int:
+    return int(lib().ogq_bucket_packed_words(int(total_elems), int(d), int(bits)))
+
+
+def ogq_clip_threshold(d_grad, d_off, T: int, total_elems: int, c: float, d_tau, d_status, d_ws, ws_bytes: int,
+                       stream=None) -> None:
+    _check(
+        lib().ogq_clip_threshold(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), float(c), _ptr(d_tau),
+                                 _ptr(d_status), _ptr(d_ws), int(ws_bytes), _stream(stream)),
+        "ogq_clip_threshold",
+    )
+
+
+def ogq_levels_orq_clipped(d_grad, d_off, T: int, total_elems: int, s: int, d_tau, d_levels, d_status, d_ws,
+                           ws_bytes: int, stream=None) -> None:
+    _check(
+        lib().ogq_levels_orq_clipped(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(s), _ptr(d_tau),
+                                     _ptr(d_levels), _ptr(d_status), _ptr(d_ws), int(ws_bytes), _stream(stream)),
+        "ogq_levels_orq_clipped",
+    )
+
+
+def ogq_levels_bingrad_clipped(d_grad, d_off, T: int, total_elems: int, variant: int, lloyd_iters: int, d_tau,
+                               d_levels, d_thresh, d_status, d_ws, ws_bytes: int, stream=None) -> None:
+    _check(
+        lib().ogq_levels_bingrad_clipped(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(variant),
+                                         int(lloyd_iters), _ptr(d_tau), _ptr(d_levels), _ptr(d_thresh),
+                                         _ptr(d_status), _ptr(d_ws), int(ws_bytes), _stream(stream)),
+        "ogq_levels_bingrad_clipped",
+    )
+
+
+def ogq_quantize_pack_clipped(d_grad, d_off, T: int, total_elems: int, scheme: int, s: int, d_levels, d_thresh,
+                              d_tau, seed: int, stream_id: int, d_packed_off, d_packed, stream=None) -> None:
+    _check(
+        lib().ogq_quantize_pack_clipped(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(scheme), int(s),
+                                        _ptr(d_levels), _ptr(d_thresh), _ptr(d_tau), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                        int(stream_id) & 0xFFFFFFFF, _ptr(d_packed_off), _ptr(d_packed),
+                                        _stream(stream)),
+        "ogq_quantize_pack_clipped",
+    )
+
+
+def ogq_bucket_encode(d_grad, total_elems: int, d: int, scheme: int, s: int, iters: int, clip_c: float, seed: int,
+                      stream_id: int, d_levels, d_thresh, d_status, d_packed, stream=None) -> None:
+    _check(
+        lib().ogq_bucket_encode(_ptr(d_grad), int(total_elems), int(d), int(scheme), int(s), int(iters), float(clip_c),
+                                int(seed) & 0xFFFFFFFFFFFFFFFF, int(stream_id) & 0xFFFFFFFF, _ptr(d_levels),
+                                _ptr(d_thresh), _ptr(d_status), _ptr(d_packed), _stream(stream)),
+        "ogq_bucket_encode",
     )
 
 

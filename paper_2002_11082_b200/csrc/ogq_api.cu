@@ -124,9 +124,10 @@ size_t ogq_workspace_bytes(int num_tensors, int64_t total_elems, int max_levels)
     return (a > b ? a : b) + 256;
 }
 
-ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
-                              int variant, int lloyd_iters, float* d_levels, float* d_thresh,
-                              int32_t* d_status, void* d_ws, size_t ws_bytes, ogq_stream_t stream)
+static ogq_status levels_bingrad_impl(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                                      int variant, int lloyd_iters, const float* d_tau, float* d_levels,
+                                      float* d_thresh, int32_t* d_status, void* d_ws, size_t ws_bytes,
+                                      ogq_stream_t stream)
 {
     if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_status || lloyd_iters < 0 ||
         lloyd_iters > 1024)
@@ -142,13 +143,46 @@ ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, 
     cudaError_t e;
     if (variant == OGQ_BINGRAD_B) {
         if (ws_bytes < ogq::ws_bytes_bingrad_b(T, total_elems)) return OGQ_ERR_WORKSPACE;
-        e = ogq::launch_levels_bingrad_b(d_grad, d_off, T, total_elems, lloyd_iters, d_levels, d_thresh,
+        e = ogq::launch_levels_bingrad_b(d_grad, d_off, T, total_elems, lloyd_iters, d_tau, d_levels, d_thresh,
                                          d_status, d_ws, sms, (cudaStream_t)stream);
     } else {
         if (ws_bytes < ogq::ws_bytes_select(T, total_elems, 2)) return OGQ_ERR_WORKSPACE;
-        e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_BINGRAD_PB, 2, d_levels, d_status,
+        e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_BINGRAD_PB, 2, d_tau, d_levels, d_status,
                                       d_ws, ws_bytes, sms, (cudaStream_t)stream);
     }
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                              int variant, int lloyd_iters, float* d_levels, float* d_thresh,
+                              int32_t* d_status, void* d_ws, size_t ws_bytes, ogq_stream_t stream)
+{
+    return levels_bingrad_impl(d_grad, d_off, T, total_elems, variant, lloyd_iters, nullptr, d_levels, d_thresh,
+                               d_status, d_ws, ws_bytes, stream);
+}
+
+ogq_status ogq_levels_bingrad_clipped(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                                      int variant, int lloyd_iters, const float* d_tau, float* d_levels,
+                                      float* d_thresh, int32_t* d_status, void* d_ws, size_t ws_bytes,
+                                      ogq_stream_t stream)
+{
+    if (!d_tau) return OGQ_ERR_INVALID_ARG;
+    return levels_bingrad_impl(d_grad, d_off, T, total_elems, variant, lloyd_iters, d_tau, d_levels, d_thresh,
+                               d_status, d_ws, ws_bytes, stream);
+}
+
+ogq_status ogq_clip_threshold(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, float c,
+                              float* d_tau, int32_t* d_status, void* d_ws, size_t ws_bytes, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_tau || !d_status || !(c > 0.f) || !(c < 1e30f))
+        return OGQ_ERR_INVALID_ARG;
+    if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
+    if (T == 0) return OGQ_OK;
+    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < ogq::ws_bytes_bingrad_b(T, total_elems)) return OGQ_ERR_WORKSPACE;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_clip_threshold(d_grad, d_off, T, total_elems, c, d_tau, d_status, d_ws, sms,
+                                               (cudaStream_t)stream);
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 
@@ -169,9 +203,9 @@ ogq_status ogq_levels_bingrad_b_noalloc(const float* d_grad, const int64_t* d_of
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 
-ogq_status ogq_levels_orq(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
-                          float* d_levels, int32_t* d_status, void* d_ws, size_t ws_bytes,
-                          ogq_stream_t stream)
+static ogq_status levels_orq_impl(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                                  const float* d_tau, float* d_levels, int32_t* d_status, void* d_ws,
+                                  size_t ws_bytes, ogq_stream_t stream)
 {
     if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_status) return OGQ_ERR_INVALID_ARG;
     if (!valid_orq_levels(s) || !select_size_ok(total_elems)) return OGQ_ERR_UNSUPPORTED;
@@ -181,14 +215,29 @@ ogq_status ogq_levels_orq(const float* d_grad, const int64_t* d_off, int T, int6
     if (ws_bytes < ogq::ws_bytes_select(T, total_elems, s)) return OGQ_ERR_WORKSPACE;
     const int sms = sm_count_of_current_device();
     if (sms <= 0) return OGQ_ERR_CUDA;
-    cudaError_t e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_ORQ, s, d_levels, d_status,
+    cudaError_t e = ogq::launch_levels_select(d_grad, d_off, T, total_elems, OGQ_ORQ, s, d_tau, d_levels, d_status,
                                               d_ws, ws_bytes, sms, (cudaStream_t)stream);
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 
-ogq_status ogq_quantize_pack(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+ogq_status ogq_levels_orq(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                          float* d_levels, int32_t* d_status, void* d_ws, size_t ws_bytes,
+                          ogq_stream_t stream)
+{
+    return levels_orq_impl(d_grad, d_off, T, total_elems, s, nullptr, d_levels, d_status, d_ws, ws_bytes, stream);
+}
+
+ogq_status ogq_levels_orq_clipped(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                                  const float* d_tau, float* d_levels, int32_t* d_status, void* d_ws,
+                                  size_t ws_bytes, ogq_stream_t stream)
+{
+    if (!d_tau) return OGQ_ERR_INVALID_ARG;
+    return levels_orq_impl(d_grad, d_off, T, total_elems, s, d_tau, d_levels, d_status, d_ws, ws_bytes, stream);
+}
+
+static ogq_status quantize_pack_impl(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
                              ogq_scheme scheme, int s, const float* d_levels, const float* d_thresh,
-                             uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
+                             const float* d_tau, uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
                              uint32_t* d_packed, ogq_stream_t stream)
 {
     if (T < 0 || total_elems < 0 || !d_off || !d_packed_off) return OGQ_ERR_INVALID_ARG;
@@ -210,9 +259,28 @@ ogq_status ogq_quantize_pack(const float* d_grad, const int64_t* d_off, int T, i
     const int sms = sm_count_of_current_device();
     if (sms <= 0) return OGQ_ERR_CUDA;
     cudaError_t e = ogq::launch_quantize_pack(d_grad, d_off, T, total_elems, (int)scheme, s, d_levels,
-                                              d_thresh, seed, stream_id, d_packed_off, d_packed, sms,
+                                              d_thresh, d_tau, seed, stream_id, d_packed_off, d_packed, sms,
                                               (cudaStream_t)stream);
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_quantize_pack(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                             ogq_scheme scheme, int s, const float* d_levels, const float* d_thresh,
+                             uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
+                             uint32_t* d_packed, ogq_stream_t stream)
+{
+    return quantize_pack_impl(d_grad, d_off, T, total_elems, scheme, s, d_levels, d_thresh, nullptr, seed,
+                              stream_id, d_packed_off, d_packed, stream);
+}
+
+ogq_status ogq_quantize_pack_clipped(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems,
+                                     ogq_scheme scheme, int s, const float* d_levels, const float* d_thresh,
+                                     const float* d_tau, uint64_t seed, uint32_t stream_id,
+                                     const int64_t* d_packed_off, uint32_t* d_packed, ogq_stream_t stream)
+{
+    if (!d_tau) return OGQ_ERR_INVALID_ARG;
+    return quantize_pack_impl(d_grad, d_off, T, total_elems, scheme, s, d_levels, d_thresh, d_tau, seed,
+                              stream_id, d_packed_off, d_packed, stream);
 }
 
 ogq_status ogq_unpack_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
@@ -229,6 +297,44 @@ ogq_status ogq_unpack_sum(const uint32_t* const* d_packed_k, const float* const*
     if (sms <= 0) return OGQ_ERR_CUDA;
     cudaError_t e = ogq::launch_unpack_sum(d_packed_k, d_levels_k, K, d_off, d_packed_off, T, total_elems, s,
                                            scale, d_out, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+int64_t ogq_bucket_packed_words(int64_t total_elems, int d, int bits)
+{
+    if (total_elems < 0 || d < 128 || d > 32768 || (d & 127) || bits < 1 || bits > 5) return -1;
+    if (total_elems == 0) return 0;
+    const int64_t nb = (total_elems + d - 1) / d;
+    const int64_t last = total_elems - (nb - 1) * d;
+    const int64_t w = (last * bits + 31) / 32;
+    return (nb - 1) * ((int64_t)d * bits / 32) + (w + 3) / 4 * 4;
+}
+
+ogq_status ogq_bucket_encode(const float* d_grad, int64_t total_elems, int d, ogq_scheme scheme, int s, int iters,
+                             float clip_c, uint64_t seed, uint32_t stream_id, float* d_levels, float* d_thresh,
+                             int32_t* d_status, uint32_t* d_packed, ogq_stream_t stream)
+{
+    if (total_elems < 0 || iters < 0 || iters > 1024 || !d_levels || !d_status || !(clip_c >= 0.f) || !(clip_c < 1e30f))
+        return OGQ_ERR_INVALID_ARG;
+    if (d < 128 || d > 32768 || (d & 127)) return OGQ_ERR_UNSUPPORTED;
+    if (scheme == OGQ_BINGRAD_B) {
+        if (s != 2) return OGQ_ERR_UNSUPPORTED;
+        if (!d_thresh) return OGQ_ERR_INVALID_ARG;
+    } else if (scheme == OGQ_BINGRAD_PB) {
+        if (s != 2) return OGQ_ERR_UNSUPPORTED;
+    } else if (scheme == OGQ_ORQ) {
+        if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
+    } else {
+        return OGQ_ERR_UNSUPPORTED;
+    }
+    if ((total_elems + d - 1) / d > 0x7fffffff) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_grad || !d_packed || !aligned16(d_grad) || !aligned16(d_packed)))
+        return OGQ_ERR_INVALID_ARG;
+    if (total_elems == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_bucket_encode(d_grad, total_elems, d, (int)scheme, s, iters, clip_c, seed, stream_id,
+                                              d_levels, d_thresh, d_status, d_packed, sms, (cudaStream_t)stream);
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 

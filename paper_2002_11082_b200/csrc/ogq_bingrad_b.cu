@@ -18,7 +18,7 @@ namespace ogq {
 
 __global__ void __launch_bounds__(kThreads)
 k_bb_pass(const float* __restrict__ grad, const int64_t* __restrict__ off, int T, int64_t total,
-          int64_t chunk, int pass, int lloyd_iters, float* __restrict__ levels,
+          int64_t chunk, int pass, int lloyd_iters, const float* __restrict__ tau_arr, float* __restrict__ levels,
           float* __restrict__ thresh, int32_t* __restrict__ status, BbWs ws)
 {
     __shared__ double sh_d[kWarps];
@@ -44,9 +44,11 @@ k_bb_pass(const float* __restrict__ grad, const int64_t* __restrict__ off, int T
     for_each_piece(off, T, lo, hi, [&](int t, int64_t tb, int64_t te, int64_t pb, int64_t pe) {
         if (pass > 0 && __ldcg(ws.done + t)) return;
         const float b0 = (pass == 0) ? -INFINITY : __ldcg(thresh + t);
+        const float tau = tau_arr ? __ldg(tau_arr + t) : INFINITY;  // clipping threshold (none: +Inf)
         double s_lo = 0.0, s_hi = 0.0;
         long long c_lo = 0;
-        visit_piece(grad, pb, pe, [&](float v) {
+        visit_piece(grad, pb, pe, [&](float raw) {
+            const float v = copysignf(fminf(fabsf(raw), tau), raw);
             const bool below = v < b0;
             const double d = (double)v;
             s_lo += below ? d : 0.0;
@@ -129,8 +131,8 @@ k_bb_pass(const float* __restrict__ grad, const int64_t* __restrict__ off, int T
 }
 
 cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, int T, int64_t total,
-                                    int lloyd_iters, float* d_levels, float* d_thresh, int32_t* d_status,
-                                    void* d_ws, int sm_count, cudaStream_t stream)
+                                    int lloyd_iters, const float* d_tau, float* d_levels, float* d_thresh,
+                                    int32_t* d_status, void* d_ws, int sm_count, cudaStream_t stream)
 {
     int target = sm_count * 4 < kMaxFlatCtas ? sm_count * 4 : kMaxFlatCtas;
     FlatGrid g = make_flat_grid(total, target, 8192);
@@ -139,7 +141,7 @@ cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, i
     if (e != cudaSuccess) return e;
     for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
         launch_begin("k_bb_pass", stream);
-        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters,
+        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, d_tau,
                                                    d_levels, d_thresh, d_status, ws);
         launch_end(stream);
     }
@@ -193,7 +195,7 @@ cudaError_t launch_levels_bingrad_b_static(const float* d_grad, const int64_t* d
     if (e != cudaSuccess) return e;
     for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
         launch_begin("k_bb_pass", stream);
-        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters,
+        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, nullptr,
                                                    d_levels, d_thresh, d_status, ws);
         launch_end(stream);
     }

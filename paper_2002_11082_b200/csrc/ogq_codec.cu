@@ -11,59 +11,16 @@
 
 #include "ogq_common.cuh"
 #include "ogq_internal.h"
+#include "ogq_quant.cuh"
 
 namespace ogq {
 
-constexpr int kMaxLevels = 32;
-constexpr int kMaxWorkers = 64;
-
-// OR-combine the 4*BITS-bit chunk of each lane into words, BITS = 1, 2 or 4: a word is made of
-// 8, 4, 2 neighbouring lanes and the first lane of each such set returns it (word index lane / L).
-template <int BITS>
-__device__ __forceinline__ uint32_t assemble_words(uint32_t chunk, int lane)
-{
-    static_assert(BITS == 1 || BITS == 2 || BITS == 4, "other widths are combined in shared memory");
-    constexpr int L = 8 / BITS;
-    uint32_t x = chunk << (4 * BITS * (lane & (L - 1)));
-#pragma unroll
-    for (int o = 1; o < L; o <<= 1) x |= __shfl_xor_sync(0xffffffffu, x, o);
-    return x;
-}
-
-// Segment search and rounding decision of one element on the fast path.  `tabaddr` is the shared
-// address of the table {level k, width of the segment above it} (8 bytes per entry) and `mid` its
-// middle level.  Returns the address of the entry whose index is the element's code: the entry of the
-// segment's lower level, or the next one when the element rounds up.  The halving steps are written
-// as "load, compare, predicated add" so that each costs three instructions.
-template <int STEP>
-__device__ __forceinline__ void search_step(uint32_t& a, float v)
-{
-    asm("{ .reg .pred p; .reg .f32 t; ld.shared.f32 t, [%0+%2]; setp.le.f32 p, t, %1; @p add.u32 %0, %0, %2; }"
-        : "+r"(a) : "f"(v), "n"(STEP * 8));
-}
-
-template <int BITS>
-__device__ __forceinline__ uint32_t entry_after_rounding(float v, uint32_t rnd, uint32_t tabaddr, float mid)
-{
-    uint32_t a = tabaddr;
-    if constexpr (BITS >= 2) {
-        if (mid <= v) a += 8u << (BITS - 2);
-        if constexpr (BITS >= 5) search_step<4>(a, v);
-        if constexpr (BITS >= 4) search_step<2>(a, v);
-        if constexpr (BITS >= 3) search_step<1>(a, v);
-    }
-    float lo, w;
-    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(lo), "=f"(w) : "r"(a));
-    const float lhs = __fmul_rn((float)(rnd >> 8), w);
-    const float rhs = __fmul_rn(__fsub_rn(v, lo), 16777216.0f);
-    asm("{ .reg .pred p; setp.lt.f32 p, %1, %2; @p add.u32 %0, %0, 8; }" : "+r"(a) : "f"(lhs), "f"(rhs));
-    return a;
-}
-
-template <int BITS, bool THRESHOLD>
+// CLIP: every value is first clamped to [-tau_arr[t], tau_arr[t]] (gradient clipping).
+template <int BITS, bool THRESHOLD, bool CLIP>
 __global__ void __launch_bounds__(kThreads)
 k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off, int T, int64_t total,
                 int64_t chunk, int s, const float* __restrict__ levels, const float* __restrict__ thresh,
+                const float* __restrict__ tau_arr,
                 const __grid_constant__ PhiloxKeys keys, uint32_t stream_id,
                 const int64_t* __restrict__ packed_off, uint32_t* __restrict__ packed)
 {
@@ -84,6 +41,8 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
         const int64_t g_beg = (pb - tb + 127) >> 7, g_end = (pe - tb + 127) >> 7;
         if (g_beg >= g_end) return;
         float b0 = 0.f;
+        const float tau = CLIP ? __ldg(tau_arr + t) : 0.f;
+        auto clip = [&](float x) -> float { return CLIP ? copysignf(fminf(fabsf(x), tau), x) : x; };
         if (THRESHOLD) {
             b0 = __ldg(thresh + t);
         } else {
@@ -132,7 +91,8 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
                     mid = sh_tab[(BITS >= 2) ? (1 << (BITS - 2)) : 0].x;
                     hz = philox_hoist(0u, (uint32_t)t, stream_id, keys);
                 }
-                auto code4 = [&](const float4 v, int gl) -> uint32_t {
+                auto code4 = [&](float4 v, int gl) -> uint32_t {
+                    if constexpr (CLIP) { v.x = clip(v.x); v.y = clip(v.y); v.z = clip(v.z); v.w = clip(v.w); }
                     if constexpr (THRESHOLD) {
                         const uint32_t b4 = ((v.x >= b0) ? 1u : 0u) | ((v.y >= b0) ? 2u : 0u) |
                                             ((v.z >= b0) ? 4u : 0u) | ((v.w >= b0) ? 8u : 0u);
@@ -184,6 +144,10 @@ k_quantize_pack(const float* __restrict__ grad, const int64_t* __restrict__ off,
             } else {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) x[j] = (i0 + j < n) ? __ldg(base + i0 + j) : 0.f;
+            }
+            if constexpr (CLIP) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) x[j] = clip(x[j]);
             }
             uint32_t c[4];
             if (THRESHOLD) {
@@ -385,16 +349,22 @@ static int flat_target(int sm_count)
 
 cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int T, int64_t total,
                                  int scheme, int s, const float* d_levels, const float* d_thresh,
-                                 uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
-                                 uint32_t* d_packed, int sm_count, cudaStream_t stream)
+                                 const float* d_tau, uint64_t seed, uint32_t stream_id,
+                                 const int64_t* d_packed_off, uint32_t* d_packed, int sm_count,
+                                 cudaStream_t stream)
 {
     FlatGrid g = make_flat_grid(total, flat_target(sm_count), 8192);
     const PhiloxKeys keys = philox_round_keys((uint32_t)seed, (uint32_t)(seed >> 32));
     const int bits = ogq_bits_for_levels(s);
-#define OGQ_LAUNCH_Q(B, TH)                                                                          \
-    k_quantize_pack<B, TH><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, s,     \
-                                                            d_levels, d_thresh, keys, stream_id,     \
-                                                            d_packed_off, d_packed)
+#define OGQ_LAUNCH_QC(B, TH, CL)                                                                        \
+    k_quantize_pack<B, TH, CL><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, s,    \
+                                                                d_levels, d_thresh, d_tau, keys,        \
+                                                                stream_id, d_packed_off, d_packed)
+#define OGQ_LAUNCH_Q(B, TH)                    \
+    do {                                       \
+        if (d_tau) OGQ_LAUNCH_QC(B, TH, true); \
+        else OGQ_LAUNCH_QC(B, TH, false);      \
+    } while (0)
     launch_begin(scheme == OGQ_BINGRAD_B ? "k_quantize_pack_threshold" : "k_quantize_pack_random", stream);
     if (scheme == OGQ_BINGRAD_B) {
         OGQ_LAUNCH_Q(1, true);
@@ -409,6 +379,7 @@ cudaError_t launch_quantize_pack(const float* d_grad, const int64_t* d_off, int 
         }
     }
 #undef OGQ_LAUNCH_Q
+#undef OGQ_LAUNCH_QC
     launch_end(stream);
     return cudaGetLastError();
 }

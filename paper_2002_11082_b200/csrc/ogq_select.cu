@@ -366,8 +366,14 @@ struct Round1Body {
                    // sums lie kCells words above the counts, their carries 2 kCells words above
     float mn, mx;
     uint32_t nonfinite;
+    float tau;  // clipping threshold (+Inf: none)
 
-    static __device__ __forceinline__ float canon(float v) { return (MAG ? fabsf(v) : v) + 0.0f; }
+    // clip to [-tau, tau], magnitude for BinGrad-pb, and fold -0 into +0
+    __device__ __forceinline__ float canon(float v) const
+    {
+        const float m = fminf(fabsf(v), tau);
+        return (MAG ? m : copysignf(m, v)) + 0.0f;
+    }
 
     // a value inside the fine window (rel = magnitude bits - lo23 < kSelW << 23)
     __device__ __forceinline__ void fine(uint32_t bits, uint32_t rel)
@@ -427,9 +433,11 @@ struct Round1Body {
 
 template <bool MAG>
 __device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe, int lo_e,
-                                              uint32_t* hist, float& vmin, float& vmax, uint32_t& nonfinite)
+                                              uint32_t* hist, float& vmin, float& vmax, uint32_t& nonfinite,
+                                              float tau)
 {
     Round1Body<MAG> f;
+    f.tau = tau;
     f.lo23 = (uint32_t)lo_e << 23;
     f.lo_e = lo_e;
     f.cnt = (uint32_t)__cvta_generic_to_shared(hist + (MAG ? 0 : kRound1Mag));
@@ -526,10 +534,14 @@ __device__ __forceinline__ void build_prefilter(Table& tb, bool magnitude_only)
     __syncthreads();
 }
 
+template <bool CLIP>
 struct Round2Warp {
     uint32_t coarse;  // shared addresses: the table's prefilter bitmap,
     uint32_t stage;   // this warp's kStageCap parking slots,
     uint32_t fillp;   // and their fill counter (bumped by the lanes that hit)
+    float tau;        // clipping threshold (CLIP only)
+
+    __device__ __forceinline__ float clip(float v) const { return CLIP ? copysignf(fminf(fabsf(v), tau), v) : v; }
 
     // Phase A for one element: no warp collective, only the lanes that pass the bitmap test do work.
     __device__ __forceinline__ void park(uint32_t bits)
@@ -545,13 +557,13 @@ struct Round2Warp {
     }
     __device__ __forceinline__ void one(float v)
     {
-        const uint32_t bits = __float_as_uint(v);
+        const uint32_t bits = __float_as_uint(clip(v));
         if (top_is_hit(bits) >> 31) park(bits);
     }
     // Branch-free form for the main loop: shifts `hits` left and appends this element's bit.
     __device__ __forceinline__ void test(float v, uint32_t& hits) const
     {
-        hits = __funnelshift_l(top_is_hit(__float_as_uint(v)), hits, 1);
+        hits = __funnelshift_l(top_is_hit(__float_as_uint(clip(v))), hits, 1);
     }
     // Parks the elements marked in `hits` (bit 7 = the first of the eight elements tested: p[0].x,
     // ..., p[0].w, p[stride].x, ...).  The values are read again, from L1: a hit is rare, and a
@@ -563,15 +575,16 @@ struct Round2Warp {
             hits &= ~(1u << b);
             const int j = 7 - b;
             const float* src = reinterpret_cast<const float*>(p + ((j & 4) ? stride : 0)) + (j & 3);
-            park(__float_as_uint(__ldg(src)));
+            park(__float_as_uint(clip(__ldg(src))));
         }
     }
 };
 
+template <bool CLIP>
 __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64_t pb, int64_t pe,
                                               bool magnitude_only, const Table& tb, uint32_t* cnt, uint32_t* lo,
                                               uint32_t* hi, uint32_t* stage, uint32_t* dst,
-                                              unsigned long long* cursor, bool nohist)
+                                              unsigned long long* cursor, bool nohist, float tau)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __shared__ Round2Ctx ctx;
@@ -584,7 +597,8 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
     }
     if (lane == 0) fills[warp] = 0;
     __syncthreads();
-    Round2Warp w;
+    Round2Warp<CLIP> w;
+    w.tau = tau;
     w.coarse = (uint32_t)__cvta_generic_to_shared(tb.coarse);
     w.stage = (uint32_t)__cvta_generic_to_shared(stage);
     w.fillp = (uint32_t)__cvta_generic_to_shared(&fills[warp]);
@@ -1523,7 +1537,7 @@ __device__ __forceinline__ int upper_bound_u32(const uint32_t* a, int n, uint32_
 
 __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, int t, int scheme, int s,
                              float* __restrict__ levels, int32_t* __restrict__ status, TState* st,
-                             unsigned char* smem)
+                             unsigned char* smem, float tau)
 {
     __shared__ double sh_d[kSelWarps];
     __shared__ uint32_t sh_lvkey[kMaxLv];
@@ -1538,7 +1552,8 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
     for (int i = threadIdx.x; i < P; i += kSelThreads) {
         uint32_t key = 0xffffffffu;
         if (i < n) {
-            uint32_t bits = __float_as_uint(__ldg(grad + tb + i));
+            const float raw = __ldg(grad + tb + i);
+            uint32_t bits = __float_as_uint(copysignf(fminf(fabsf(raw), tau), raw));
             if ((bits & 0x7f800000u) == 0x7f800000u) sh_flag = 1;
             if (pb) key = bits | 0x80000000u;
             else {
@@ -1642,6 +1657,7 @@ __device__ void small_tensor(const float* __restrict__ grad, int64_t tb, int n, 
 // ---------------------------------------------------------------------------
 struct SelArgs {
     const float* grad;
+    const float* tau;  // per-tensor clipping thresholds, or null
     const int64_t* off;
     int T;
     int64_t total, chunk;
@@ -1739,6 +1755,7 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         TState* st = A.ws.st + t;
         const int hi_e = window_anchor(tbeg, n);
         const int lo_e = hi_e - kSelW;
+        const float tau = A.tau ? __ldg(A.tau + t) : __int_as_float(0x7f800000);
         const int ncells = pb ? kRound1Mag : kRound1Cells;
         uint32_t* gcnt = A.ws.gcnt + (size_t)t * kCells;
         unsigned long long* glsum = A.ws.glsum + (size_t)t * kCells;
@@ -1746,8 +1763,8 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         uint32_t nf = 0u;
         zero_hist(hist, ncells);
         __syncthreads();
-        if (pb) stream_round1<true>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf);
-        else stream_round1<false>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf);
+        if (pb) stream_round1<true>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf, tau);
+        else stream_round1<false>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf, tau);
         __syncthreads();
         // The low sums of the window's cells are 32 bits wide without a carry: exact as long as no such
         // cell took more than 2^16 values.  Otherwise (heavily repeated values) the piece is redone in
@@ -1765,8 +1782,8 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
                 const int64_t qe = (q + kR1MaxPiece < pe_) ? q + kR1MaxPiece : pe_;
                 zero_hist(hist, ncells);
                 __syncthreads();
-                if (pb) stream_round1<true>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf);
-                else stream_round1<false>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf);
+                if (pb) stream_round1<true>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf, tau);
+                else stream_round1<false>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf, tau);
                 __syncthreads();
                 flush_hist(hist, ncells, gcnt, glsum);
                 __syncthreads();
@@ -1849,7 +1866,8 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
             if (threadIdx.x < nl) A.levels[(int64_t)t * nl + threadIdx.x] = 0.f;
             if (threadIdx.x == 0) { A.status[t] = OGQ_ST_EMPTY; A.ws.st[t].done = 1; }
         } else if (n <= kSmallN) {
-            small_tensor(A.grad, tbeg, (int)n, t, A.scheme, A.s, A.levels, A.status, A.ws.st + t, smem);
+            small_tensor(A.grad, tbeg, (int)n, t, A.scheme, A.s, A.levels, A.status, A.ws.st + t, smem,
+                         A.tau ? __ldg(A.tau + t) : __int_as_float(0x7f800000));
         } else if (n <= kMidN) {
             // round 1 and its solver pass on this CTA; the tensor's CTA of the round-2 kernel goes on from there
             r1_stream(t, tbeg, tend, tbeg, tend, true);
@@ -1903,9 +1921,13 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
         copy_only = __ldcg(&st->compact_only) != 0;
         if (!copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
-        stream_round2(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells,
-                      reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap,
-                      A.ws.buf[0] + tbeg, &st->cursor[0], copy_only);
+        uint32_t* stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+        if (A.tau)
+            stream_round2<true>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stage,
+                                A.ws.buf[0] + tbeg, &st->cursor[0], copy_only, __ldg(A.tau + t));
+        else
+            stream_round2<false>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stage,
+                                 A.ws.buf[0] + tbeg, &st->cursor[0], copy_only, 0.f);
         __syncthreads();
         if (!copy_only) flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         __threadfence();
@@ -2037,8 +2059,8 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
 }
 
 cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int T, int64_t total, int scheme,
-                                 int s, float* d_levels, int32_t* d_status, void* d_ws, size_t /*ws_bytes*/,
-                                 int sm_count, cudaStream_t stream)
+                                 int s, const float* d_tau, float* d_levels, int32_t* d_status, void* d_ws,
+                                 size_t /*ws_bytes*/, int sm_count, cudaStream_t stream)
 {
     {
         // the kernels need more dynamic shared memory than the default limit: raised once per device
@@ -2064,7 +2086,7 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     const int target = wave < kMaxFlatCtas ? (int)wave : kMaxFlatCtas;
     FlatGrid g = make_flat_grid(total, target, 32768);
     SelArgs A;
-    A.grad = d_grad; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
+    A.grad = d_grad; A.tau = d_tau; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
     A.scheme = scheme; A.s = s; A.levels = d_levels; A.status = d_status;
     A.ws = sel_carve(d_ws, T, total);
     cudaError_t e = cudaMemsetAsync(d_ws, 0, sel_zero_bytes(T), stream);

@@ -39,7 +39,7 @@ class DeviceBucket:
         torch.cuda.synchronize()
         return lv.cpu().numpy(), st.cpu().numpy()
 
-    def quantize_pack(self, scheme: int, s: int, levels, thresh, seed: int, stream_id: int):
+    def quantize_pack(self, scheme: int, s: int, levels, thresh, seed: int, stream_id: int, tau=None):
         bits = ogq.ogq_bits_for_levels(s)
         h_po = ogq.ogq_packed_layout(self.h_off, bits)
         po = torch.from_numpy(h_po).to(self.dev)
@@ -49,7 +49,11 @@ class DeviceBucket:
         packed = buf[pad : pad + int(h_po[-1])]
         d_lv = torch.from_numpy(np.ascontiguousarray(levels, dtype=np.float32)).to(self.dev) if levels is not None else None
         d_th = torch.from_numpy(np.ascontiguousarray(thresh, dtype=np.float32)).to(self.dev) if thresh is not None else None
-        ogq.ogq_quantize_pack(self.grad, self.off, self.T, self.N, scheme, s, d_lv, d_th, seed, stream_id, po, packed)
+        if tau is None:
+            ogq.ogq_quantize_pack(self.grad, self.off, self.T, self.N, scheme, s, d_lv, d_th, seed, stream_id, po, packed)
+        else:
+            ogq.ogq_quantize_pack_clipped(self.grad, self.off, self.T, self.N, scheme, s, d_lv, d_th, tau, seed,
+                                          stream_id, po, packed)
         torch.cuda.synchronize()
         h = buf.cpu().numpy().view(np.uint32)
         assert np.all(h[:pad] == 0x5A5A5A5A) and np.all(h[pad + int(h_po[-1]) :] == 0x5A5A5A5A), "canary overwritten"
