@@ -246,7 +246,7 @@ def stored_traffic(kernel: str, scheme: str):
 class Setup:
     """One workload x scheme resident in HBM: K workers' buckets, outputs, scratch, streams."""
 
-    def __init__(self, torch, ogq, dev, workload, scheme_name, K, seed, rank, bucket_len=0, share=None):
+    def __init__(self, torch, ogq, dev, workload, scheme_name, K, seed, rank, bucket_len=0, share=None, dense=False):
         from paper_2002_11082_b200.sharding import worker_ids
 
         self.torch, self.ogq, self.dev = torch, ogq, dev
@@ -255,6 +255,7 @@ class Setup:
         self.bits = ogq.ogq_bits_for_levels(self.s)
         self.bucket_len = bucket_len
         self.clip_c = 0.0
+        self.dense = bool(dense) and self.scheme == 2
         if share is not None and share.workload == workload:
             self.host, self.grads = share.host, share.grads
         else:
@@ -269,7 +270,8 @@ class Setup:
         self.T = self.h_off.size - 1
         T, s = self.T, self.s
         self.off = torch.from_numpy(self.h_off).to(dev)
-        self.h_po = ogq.ogq_packed_layout(self.h_off, self.bits)
+        self.h_po = ogq.ogq_dense_layout(self.h_off, self.s) if self.dense else ogq.ogq_packed_layout(self.h_off, self.bits)
+        self.code_bits = 32.0 / ogq.ogq_dense_digits(self.s) if self.dense else float(self.bits)
         self.po = torch.from_numpy(self.h_po).to(dev)
         self.levels = [torch.zeros((T, s), device=dev) for _ in range(K)]
         self.thresh = [torch.zeros((T,), device=dev) for _ in range(K)]
@@ -282,7 +284,7 @@ class Setup:
         self.pk_ptrs = ogq.device_pointer_array(self.packed)
         self.lv_ptrs = ogq.device_pointer_array(self.levels)
         self.grad_bytes = 4.0 * self.N * K
-        self.alg_lqp = (8.0 + self.bits / 8.0) * self.N * K
+        self.alg_lqp = (8.0 + self.code_bits / 8.0) * self.N * K
 
     def lqp(self, k, stream=None, slot=None):
         """levels + quantize + pack of worker k (scratch slot = the stream's own)."""
@@ -294,8 +296,12 @@ class Setup:
         elif self.scheme == ogq.OGQ_ORQ:
             ogq.ogq_levels_orq(self.grads[k], self.off, self.T, self.N, s, self.levels[k], self.status[k], ws,
                                self.ws_bytes, stream)
-            ogq.ogq_quantize_pack(self.grads[k], self.off, self.T, self.N, self.scheme, s, self.levels[k], None,
-                                  self.seed, k, self.po, self.packed[k], stream)
+            if self.dense:
+                ogq.ogq_quantize_pack_dense(self.grads[k], self.off, self.T, self.N, s, self.levels[k], self.seed, k,
+                                            self.po, self.packed[k], stream)
+            else:
+                ogq.ogq_quantize_pack(self.grads[k], self.off, self.T, self.N, self.scheme, s, self.levels[k], None,
+                                      self.seed, k, self.po, self.packed[k], stream)
         else:
             ogq.ogq_levels_bingrad(self.grads[k], self.off, self.T, self.N, self.scheme, self.lloyd, self.levels[k],
                                    self.thresh[k], self.status[k], ws, self.ws_bytes, stream)
@@ -303,6 +309,10 @@ class Setup:
                                   self.thresh[k], self.seed, k, self.po, self.packed[k], stream)
 
     def unpack(self):
+        if self.dense:
+            self.ogq.ogq_unpack_sum_dense(self.pk_ptrs, self.lv_ptrs, self.K, self.off, self.po, self.T, self.N, self.s,
+                                          1.0 / self.K, self.out)
+            return
         self.ogq.ogq_unpack_sum(self.pk_ptrs, self.lv_ptrs, self.K, self.off, self.po, self.T, self.N, self.s,
                                 1.0 / self.K, self.out)
 
@@ -395,8 +405,8 @@ def run_ours(args):
         barrier()
         return max_over_ranks(total, dist, dev)
 
-    S = Setup(torch, ogq, dev, args.workload, args.scheme, K, args.seed, rank, args.bucket_len)
-    N, T, bits, s = S.N, S.T, S.bits, S.s
+    S = Setup(torch, ogq, dev, args.workload, args.scheme, K, args.seed, rank, args.bucket_len, dense=args.dense)
+    N, T, bits, s = S.N, S.T, S.code_bits, S.s
     # L2 hygiene: the large buckets cycle through far more than the 126 MB L2 per step
     need_flush = 4 * N * K <= 2 * 126e6
 
@@ -425,7 +435,7 @@ def run_ours(args):
         ms = timed(lambda: setup.lqp_all(streams), reps, flush) / reps
         gbs = setup.alg_lqp / (ms * 1e-3) / 1e9
         return {"streams": streams, "ms": ms, "grad_gbs": setup.grad_bytes / (ms * 1e-3) / 1e9,
-                "alg_bytes_per_elem": 8.0 + setup.bits / 8.0, "frac_of_hbm_peak": gbs / peak,
+                "alg_bytes_per_elem": 8.0 + setup.code_bits / 8.0, "frac_of_hbm_peak": gbs / peak,
                 "frac_of_nominal_8tbs": gbs / 8000.0}
 
     # ---- per-stage and per-kernel times (separate instrumented passes, not part of `value`)
@@ -448,6 +458,7 @@ def run_ours(args):
         "k_sel_round1": 4.0 * N, "k_sel_round2": 4.0 * N, "k_sel_round3": 0.0, "k_bb_pass": 4.0 * N,
         "k_quantize_pack_random": (4.0 + bits / 8.0) * N, "k_quantize_pack_threshold": (4.0 + 1 / 8.0) * N,
         "k_unpack_sum": (K * bits / 8.0 + 4.0) * N, "k_bucket_encode": (4.0 + bits / 8.0) * N,
+        "k_quantize_pack_dense": (4.0 + bits / 8.0) * N, "k_unpack_sum_dense": (K * bits / 8.0 + 4.0) * N,
     }
     kernels = {}
     total_ms = max(sum(v[0] for v in per_kernel.values()), 1e-12)
@@ -515,7 +526,7 @@ def run_ours(args):
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "scheme": args.scheme, "levels": s, "bits": bits,
                        "workers_per_gpu": K, "tensors": T, "elements": N, "streams": n_streams,
-                       "bucket_len": args.bucket_len or None,
+                       "bucket_len": args.bucket_len or None, "packing": "base-s words" if S.dense else "bit stream",
                        "l2": "256 MB written between timed steps (flush)" if need_flush else "inputs larger than L2 (no flush)"},
             "stages": {
                 "levels_quantize_pack": st_multi,
@@ -545,6 +556,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-secondary", action="store_true")
+    ap.add_argument("--dense", action="store_true", help="ORQ codes in the base-s (entropy-dense) wire format")
     ap.add_argument("--bucket-len", type=int, default=0,
                     help="fixed-length bucket mode: quantize buckets of this many elements (ogq_bucket_encode)")
     args = ap.parse_args()

@@ -173,6 +173,46 @@ ogq_status ogq_unpack_sum(const uint32_t *const *d_packed_k, const float *const 
                           int s, float scale, float *d_out, ogq_stream_t stream);
 
 /*
+ * Quantization error per tensor, d_err [T] in fp64 (a diagnostic, not on the encode path).
+ *   ogq_quant_error: the realised error of bit-packed codes, sum_i (levels[code_i] - v_i)^2,
+ *     the ||Q(G) - G||^2 the paper records during training (Section "Performance" of the CIFAR
+ *     experiments and its training-curve figure).  s = 2 decodes 1-bit codes of either BinGrad.
+ *   ogq_expected_error: its expectation over the random rounding, sum_i (v_i - lo_i)(hi_i - v_i)
+ *     with lo, hi the levels around v_i (the functional in the proof of Theorem 1); a value
+ *     outside the levels counts with its squared distance to the end level.
+ * Sums are fp64 per thread, combined with one fp64 atomic per CTA and tensor piece: the last
+ * bits can differ from run to run.
+ */
+ogq_status ogq_quant_error(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems, int s,
+                           const float *d_levels, const int64_t *d_packed_off, const uint32_t *d_packed,
+                           double *d_err, ogq_stream_t stream);
+ogq_status ogq_expected_error(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems, int s,
+                              const float *d_levels, double *d_err, ogq_stream_t stream);
+
+/*
+ * Entropy-dense wire format (Tables of the CIFAR-100 and ImageNet results: compression ratios
+ * x20.2, x13.8, x10.1 for 3, 5, 9 levels, i.e. 32 / log2(s): a code is taken to cost log2(s)
+ * bits).  The closest whole-word format: M consecutive codes of a tensor are the base-s digits,
+ * least significant first, of one 32-bit word, M = ogq_dense_digits(s) the largest count with
+ * s^M <= 2^32 (s = 3: 20, 5: 13, 9: 10, 17: 7; 0 for other s), so ratios x20 / x13 / x10 / x7
+ * against x16 / x10.7 / x8 / x6.4 of the bit-packed format.  Word j of a tensor holds elements
+ * j M ... j M + M - 1, missing elements count as code 0, and regions are zero padded to a
+ * multiple of 4 words (ogq_dense_layout, host-only, fills h_packed_off[0..T]).
+ *   ogq_quantize_pack_dense: the ORQ quantizer of ogq_quantize_pack (same segment search, same
+ *     Philox counters, same rounding decision, hence the same codes), packed in this format.
+ *   ogq_unpack_sum_dense: ogq_unpack_sum for this format.
+ */
+int ogq_dense_digits(int s);
+ogq_status ogq_dense_layout(const int64_t *h_off, int T, int s, int64_t *h_packed_off);
+ogq_status ogq_quantize_pack_dense(const float *d_grad, const int64_t *d_off, int T, int64_t total_elems,
+                                   int s, const float *d_levels, uint64_t seed, uint32_t stream_id,
+                                   const int64_t *d_packed_off, uint32_t *d_packed, ogq_stream_t stream);
+ogq_status ogq_unpack_sum_dense(const uint32_t *const *d_packed_k, const float *const *d_levels_k, int K,
+                                const int64_t *d_off, const int64_t *d_packed_off, int T,
+                                int64_t total_elems, int s, float scale, float *d_out,
+                                ogq_stream_t stream);
+
+/*
  * Gradient clipping (Section "Experiments", paragraph after the list of methods):
  * clip(v) = sign(v) min(|v|, c sigma), sigma^2 the variance of the gradient being quantized
  * (here: of each tensor, about its mean, over all its elements), c = 2.5 in the ImageNet runs,

@@ -27,6 +27,12 @@ from .binding import (  # noqa: F401
     ogq_levels_orq,
     ogq_quantize_pack,
     ogq_unpack_sum,
+    ogq_quant_error,
+    ogq_expected_error,
+    ogq_dense_digits,
+    ogq_dense_layout,
+    ogq_quantize_pack_dense,
+    ogq_unpack_sum_dense,
     ogq_clip_threshold,
     ogq_levels_orq_clipped,
     ogq_levels_bingrad_clipped,

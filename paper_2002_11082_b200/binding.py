@@ -68,6 +68,18 @@ def lib() -> ctypes.CDLL:
         L.ogq_clip_threshold.argtypes = [vp, vp, i32, i64, ctypes.c_float, vp, vp, vp, sz, vp]
         L.ogq_levels_orq_clipped.restype = i32
         L.ogq_levels_orq_clipped.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, sz, vp]
+        L.ogq_quant_error.restype = i32
+        L.ogq_quant_error.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, vp]
+        L.ogq_expected_error.restype = i32
+        L.ogq_expected_error.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+        L.ogq_dense_digits.restype = i32
+        L.ogq_dense_digits.argtypes = [i32]
+        L.ogq_dense_layout.restype = i32
+        L.ogq_dense_layout.argtypes = [vp, i32, i32, vp]
+        L.ogq_quantize_pack_dense.restype = i32
+        L.ogq_quantize_pack_dense.argtypes = [vp, vp, i32, i64, i32, vp, ctypes.c_uint64, ctypes.c_uint32, vp, vp, vp]
+        L.ogq_unpack_sum_dense.restype = i32
+        L.ogq_unpack_sum_dense.argtypes = [vp, vp, i32, vp, vp, i32, i64, i32, ctypes.c_float, vp, vp]
         L.ogq_quantize_pack_clipped.restype = i32
         L.ogq_quantize_pack_clipped.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, ctypes.c_uint64, ctypes.c_uint32,
                                                 vp, vp, vp]
@@ -208,6 +220,54 @@ def ogq_levels_bingrad_clipped(d_grad, d_off, T: int, total_elems: int, variant:
                                          int(lloyd_iters), _ptr(d_tau), _ptr(d_levels), _ptr(d_thresh),
                                          _ptr(d_status), _ptr(d_ws), int(ws_bytes), _stream(stream)),
         "ogq_levels_bingrad_clipped",
+    )
+
+
+def ogq_quant_error(d_grad, d_off, T: int, total_elems: int, s: int, d_levels, d_packed_off, d_packed, d_err,
+                    stream=None) -> None:
+    _check(
+        lib().ogq_quant_error(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(s), _ptr(d_levels),
+                              _ptr(d_packed_off), _ptr(d_packed), _ptr(d_err), _stream(stream)),
+        "ogq_quant_error",
+    )
+
+
+def ogq_expected_error(d_grad, d_off, T: int, total_elems: int, s: int, d_levels, d_err, stream=None) -> None:
+    _check(
+        lib().ogq_expected_error(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(s), _ptr(d_levels),
+                                 _ptr(d_err), _stream(stream)),
+        "ogq_expected_error",
+    )
+
+
+def ogq_dense_digits(s: int) -> int:
+    return int(lib().ogq_dense_digits(int(s)))
+
+
+def ogq_dense_layout(h_off, s: int) -> np.ndarray:
+    """Host helper: word offsets [T+1] of the base-s packed regions for element offsets h_off [T+1]."""
+    h = np.ascontiguousarray(np.asarray(h_off), dtype=np.int64)
+    out = np.zeros_like(h)
+    _check(lib().ogq_dense_layout(h.ctypes.data, h.size - 1, int(s), out.ctypes.data), "ogq_dense_layout")
+    return out
+
+
+def ogq_quantize_pack_dense(d_grad, d_off, T: int, total_elems: int, s: int, d_levels, seed: int, stream_id: int,
+                            d_packed_off, d_packed, stream=None) -> None:
+    _check(
+        lib().ogq_quantize_pack_dense(_ptr(d_grad), _ptr(d_off), int(T), int(total_elems), int(s), _ptr(d_levels),
+                                      int(seed) & 0xFFFFFFFFFFFFFFFF, int(stream_id) & 0xFFFFFFFF,
+                                      _ptr(d_packed_off), _ptr(d_packed), _stream(stream)),
+        "ogq_quantize_pack_dense",
+    )
+
+
+def ogq_unpack_sum_dense(d_packed_k, d_levels_k, K: int, d_off, d_packed_off, T: int, total_elems: int, s: int,
+                         scale: float, d_out, stream=None) -> None:
+    _check(
+        lib().ogq_unpack_sum_dense(_ptr(d_packed_k), _ptr(d_levels_k), int(K), _ptr(d_off), _ptr(d_packed_off),
+                                   int(T), int(total_elems), int(s), float(scale), _ptr(d_out), _stream(stream)),
+        "ogq_unpack_sum_dense",
     )
 
 

@@ -300,6 +300,85 @@ ogq_status ogq_unpack_sum(const uint32_t* const* d_packed_k, const float* const*
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 
+static ogq_status quant_error_impl(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                                   const float* d_levels, const int64_t* d_packed_off, const uint32_t* d_packed,
+                                   bool realised, double* d_err, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_err) return OGQ_ERR_INVALID_ARG;
+    if (realised && (!d_packed_off || (total_elems > 0 && !d_packed))) return OGQ_ERR_INVALID_ARG;
+    if (!(s == 2 || valid_orq_levels(s))) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && !d_grad) return OGQ_ERR_INVALID_ARG;
+    if (T == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_quant_error(d_grad, d_off, T, total_elems, s, d_levels, d_packed_off,
+                                            realised ? d_packed : nullptr, d_err, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_quant_error(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                           const float* d_levels, const int64_t* d_packed_off, const uint32_t* d_packed,
+                           double* d_err, ogq_stream_t stream)
+{
+    return quant_error_impl(d_grad, d_off, T, total_elems, s, d_levels, d_packed_off, d_packed, true, d_err, stream);
+}
+
+ogq_status ogq_expected_error(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                              const float* d_levels, double* d_err, ogq_stream_t stream)
+{
+    return quant_error_impl(d_grad, d_off, T, total_elems, s, d_levels, nullptr, nullptr, false, d_err, stream);
+}
+
+int ogq_dense_digits(int s) { return ogq::dense_digits(s); }
+
+ogq_status ogq_dense_layout(const int64_t* h_off, int T, int s, int64_t* h_packed_off)
+{
+    const int m = ogq::dense_digits(s);
+    if (!h_off || !h_packed_off || T < 0) return OGQ_ERR_INVALID_ARG;
+    if (m == 0) return OGQ_ERR_UNSUPPORTED;
+    h_packed_off[0] = 0;
+    for (int t = 0; t < T; ++t) {
+        const int64_t n = h_off[t + 1] - h_off[t];
+        if (n < 0) return OGQ_ERR_INVALID_ARG;
+        const int64_t w = (n + m - 1) / m;
+        h_packed_off[t + 1] = h_packed_off[t] + (w + 3) / 4 * 4;
+    }
+    return OGQ_OK;
+}
+
+ogq_status ogq_quantize_pack_dense(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
+                                   const float* d_levels, uint64_t seed, uint32_t stream_id,
+                                   const int64_t* d_packed_off, uint32_t* d_packed, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_packed_off || !d_levels) return OGQ_ERR_INVALID_ARG;
+    if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_grad || !d_packed || !aligned16(d_grad) || !aligned16(d_packed)))
+        return OGQ_ERR_INVALID_ARG;
+    if (T == 0 || total_elems == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_quantize_pack_dense(d_grad, d_off, T, total_elems, s, d_levels, seed, stream_id,
+                                                    d_packed_off, d_packed, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_unpack_sum_dense(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                                const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total_elems,
+                                int s, float scale, float* d_out, ogq_stream_t stream)
+{
+    if (T < 0 || total_elems < 0 || !d_off || !d_packed_off || !d_packed_k || !d_levels_k)
+        return OGQ_ERR_INVALID_ARG;
+    if (K < 1 || K > 64) return OGQ_ERR_INVALID_ARG;
+    if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_out || !aligned16(d_out))) return OGQ_ERR_INVALID_ARG;
+    if (T == 0 || total_elems == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_unpack_sum_dense(d_packed_k, d_levels_k, K, d_off, d_packed_off, T, total_elems, s,
+                                                 scale, d_out, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
 int64_t ogq_bucket_packed_words(int64_t total_elems, int d, int bits)
 {
     if (total_elems < 0 || d < 128 || d > 32768 || (d & 127) || bits < 1 || bits > 5) return -1;

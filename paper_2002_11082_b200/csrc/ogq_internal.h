@@ -46,4 +46,17 @@ cudaError_t launch_bucket_encode(const float* d_grad, int64_t total, int d, int 
                                  float clip_c, uint64_t seed, uint32_t stream_id, float* d_levels, float* d_thresh,
                                  int32_t* d_status, uint32_t* d_packed, int sm_count, cudaStream_t stream);
 
+// d_packed null: expected error of random rounding; else the realised error of those codes
+cudaError_t launch_quant_error(const float* d_grad, const int64_t* d_off, int T, int64_t total, int s,
+                               const float* d_levels, const int64_t* d_packed_off, const uint32_t* d_packed,
+                               double* d_err, int sm_count, cudaStream_t stream);
+int dense_digits(int s);  // codes per 32-bit word of the base-s format (0: unsupported s)
+cudaError_t launch_quantize_pack_dense(const float* d_grad, const int64_t* d_off, int T, int64_t total, int s,
+                                       const float* d_levels, uint64_t seed, uint32_t stream_id,
+                                       const int64_t* d_packed_off, uint32_t* d_packed, int sm_count,
+                                       cudaStream_t stream);
+cudaError_t launch_unpack_sum_dense(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                                    const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total, int s,
+                                    float scale, float* d_out, int sm_count, cudaStream_t stream);
+
 }  // namespace ogq
