@@ -537,6 +537,8 @@ static int bkt_pow2(int d)
 }
 
 // keys per thread of the register sort: 4 for the shortest buckets, 32 for the longest, else 16
+// (measured on 512- and 2048-element buckets: 16 keys per thread beat 8 and 4, although fewer
+// warps are resident: the stages that stay in registers are the cheapest)
 static int bkt_kpt(int d)
 {
     const int P = bkt_pow2(d);

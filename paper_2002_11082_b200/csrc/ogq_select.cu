@@ -48,6 +48,7 @@ static_assert(kRound1Cells <= kCells, "round-1 cells exceed the budget");
 struct TState {
     int done, round, m, hi_e;
     unsigned kmin_inv, kmax, nonfinite, arrive;
+    unsigned long long arrived;  // elements of the current pass whose counts have been flushed
     unsigned expected;
     int compact_only;  // the next pass only copies the keys inside the intervals: they fit one sort
     unsigned long long cursor[2];
@@ -325,12 +326,6 @@ __device__ __forceinline__ void visit_plain(const float* __restrict__ grad, int6
     }
 }
 
-// Round 1 over grad[pb, pe).  Per element two shared atomics without a return value: the cell's
-// count and the sum of its low key bits.  Inside the fine window the low bits are below 2^16 and a
-// CTA flushes its cells at least every kR1MaxPiece = 2^16 elements, so that sum cannot overflow 32
-// bits; only the rare values outside the window (23 low bits) go through the carry word.  Min and
-// max are tracked as floats; -0 is folded into +0 by adding +0 first.
-constexpr int64_t kR1MaxPiece = (int64_t)1 << 16;
 
 __device__ __forceinline__ float min3f(float a, float b, float c)
 {
@@ -358,40 +353,72 @@ __device__ __forceinline__ uint32_t atom_shared_add(uint32_t addr, uint32_t v)
     return old;
 }
 
-template <bool MAG>
+constexpr int kPackedPerSign = kSelW << kSelM;  // fine cells per sign (2048)
+constexpr int kPackedCells = 2 * kPackedPerSign;
+constexpr int kPackTrips = 4;                    // loop trips between two folds of the packed cells
+static_assert(kPackedCells * sizeof(uint32_t) <= kSelWarps * kStageCap * sizeof(uint32_t),
+              "the packed cells live in the (otherwise unused) compaction stages during round 1");
+
+template <bool MAG, bool CLIP>
 struct Round1Body {
     uint32_t lo23;
+    uint32_t neg_lo23x2;  // -(lo23 << 1), the addend of the doubled window offset
     int lo_e;
     uint32_t cnt;  // shared address of the count of the first non-negative magnitude cell; the low
                    // sums lie kCells words above the counts, their carries 2 kCells words above
+    uint32_t pk;   // shared address of the packed words: kPackedPerSign cells of the non-negative values,
+                   // then (signed keys only) kPackedPerSign cells of the negative ones, both by magnitude
+    uint32_t coarse;  // shared address of the counter of values that bypassed the packed cells
+    uint32_t one24;   // 1 << 24 (the count field of a packed word), kept in a register
     float mn, mx;
     uint32_t nonfinite;
-    float tau;  // clipping threshold (+Inf: none)
+    float tau;  // clipping threshold (CLIP only)
 
-    // clip to [-tau, tau], magnitude for BinGrad-pb, and fold -0 into +0
+    // clip to [-tau, tau] (CLIP), magnitude for BinGrad-pb, and fold -0 into +0
     __device__ __forceinline__ float canon(float v) const
     {
-        const float m = fminf(fabsf(v), tau);
-        return (MAG ? m : copysignf(m, v)) + 0.0f;
+        if (CLIP) {
+            const float m = fminf(fabsf(v), tau);
+            return (MAG ? m : copysignf(m, v)) + 0.0f;
+        }
+        return (MAG ? fabsf(v) : v) + 0.0f;
     }
 
-    // a value inside the fine window (rel = magnitude bits - lo23 < kSelW << 23)
-    __device__ __forceinline__ void fine(uint32_t bits, uint32_t rel)
+    // A value inside the fine window, the slow way: two adds into the wide counters (cells and low bits
+    // mirrored for negative values, so that both ascend with the key).  rel = magnitude bits - lo23.
+    __device__ __forceinline__ void fine_wide(uint32_t bits, uint32_t rel)
     {
         const int sgn = MAG ? 0 : ((int)bits >> 31);  // 0 or -1
+        const uint32_t low = (bits ^ (uint32_t)sgn) & ((1u << (23 - kSelM)) - 1u);
         const uint32_t c = cnt + (uint32_t)(((lo_e + (int)(rel >> (23 - kSelM))) ^ sgn) << 2);
         red_shared_add(c, 1u);
-        red_shared_add(c + 4u * kCells, (bits ^ (uint32_t)sgn) & ((1u << (23 - kSelM)) - 1u));
+        const uint32_t old = atom_shared_add(c + 4u * kCells, low);
+        if (old + low < old) red_shared_add(c + 8u * kCells, 1u);
+    }
+
+    // The fast way: one shared-memory add of {count 1 in the top 8 bits, low magnitude bits in the other
+    // 24} into the cell's packed word (r2 = rel << 1, below kSelW << 24).  The caller folds the packed
+    // words into the wide counters every few trips, before a cell can have taken 256 values (and redoes
+    // the trips the slow way if one did); the mirroring of the negative half happens there.  The
+    // instruction mix matters here: the loop is bound by the integer/logic pipe, so the address is put
+    // together with multiply-adds and the sign is not branched on.
+    __device__ __forceinline__ void fine_packed(uint32_t bits, uint32_t r2)
+    {
+        uint32_t addr = pk + ((r2 >> (24 - kSelM - 2)) & ((uint32_t)(kPackedPerSign - 1) << 2));
+        if (!MAG) asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(addr) : "r"(bits >> 31), "r"(4u * kPackedPerSign));
+        red_shared_add(addr, (bits & ((1u << (23 - kSelM)) - 1u)) | one24);
     }
 
     // any value (already canonical)
+    template <bool PACKED>
     __device__ __forceinline__ void any(uint32_t bits)
     {
         const int sgn = MAG ? 0 : ((int)bits >> 31);
         const uint32_t mag = bits & 0x7fffffffu;
         const uint32_t rel = mag - lo23;
         if (rel < ((uint32_t)kSelW << 23)) {
-            fine(bits, rel);
+            if (PACKED) fine_packed(bits, rel << 1);
+            else fine_wide(bits, rel);
         } else {  // outside the fine window: one cell per binade
             const int e = (int)(mag >> 23);
             const int mi = (e < lo_e) ? e : e - kSelW + (kSelW << kSelM);
@@ -401,6 +428,7 @@ struct Round1Body {
             red_shared_add(c, 1u);
             const uint32_t old = atom_shared_add(c + 4u * kCells, low);
             if (old + low < old) red_shared_add(c + 8u * kCells, 1u);
+            if (PACKED) red_shared_add(coarse, 1u);
         }
     }
 
@@ -409,9 +437,10 @@ struct Round1Body {
         v = canon(v);
         mn = fminf(mn, v);
         mx = fmaxf(mx, v);
-        any(__float_as_uint(v));
+        any<false>(__float_as_uint(v));
     }
 
+    template <bool PACKED>
     __device__ __forceinline__ void four(float4 x)
     {
         const float v0 = canon(x.x), v1 = canon(x.y), v2 = canon(x.z), v3 = canon(x.w);
@@ -419,28 +448,49 @@ struct Round1Body {
         mx = max3f(max3f(mx, v0, v1), v2, v3);
         const uint32_t b0 = __float_as_uint(v0), b1 = __float_as_uint(v1), b2 = __float_as_uint(v2),
                        b3 = __float_as_uint(v3);
-        const uint32_t r0 = (b0 & 0x7fffffffu) - lo23, r1 = (b1 & 0x7fffffffu) - lo23,
-                       r2 = (b2 & 0x7fffffffu) - lo23, r3 = (b3 & 0x7fffffffu) - lo23;
-        // the window spans kSelW = 2^4 binades, so "all four inside" is one test on the OR
+        // doubled offset into the window, (magnitude bits - lo23) << 1: the doubling drops the sign bit,
+        // and a multiply-add does both steps outside the integer/logic pipe
+        uint32_t r0, r1, r2, r3;
+        asm("mad.lo.u32 %0, %1, 2, %2;" : "=r"(r0) : "r"(b0), "r"(neg_lo23x2));
+        asm("mad.lo.u32 %0, %1, 2, %2;" : "=r"(r1) : "r"(b1), "r"(neg_lo23x2));
+        asm("mad.lo.u32 %0, %1, 2, %2;" : "=r"(r2) : "r"(b2), "r"(neg_lo23x2));
+        asm("mad.lo.u32 %0, %1, 2, %2;" : "=r"(r3) : "r"(b3), "r"(neg_lo23x2));
+        // the window spans kSelW = 2^4 binades, so "all four inside" is one test on the OR (a value
+        // below the window wraps to at least kSelW << 24 as well, because lo23 < 2^31 - 2^27)
         static_assert((kSelW & (kSelW - 1)) == 0, "window size must be a power of two");
-        if ((r0 | r1 | r2 | r3) < ((uint32_t)kSelW << 23)) {
-            fine(b0, r0); fine(b1, r1); fine(b2, r2); fine(b3, r3);
+        if ((r0 | r1 | r2 | r3) < ((uint32_t)kSelW << 24)) {
+            if (PACKED) {
+                fine_packed(b0, r0); fine_packed(b1, r1); fine_packed(b2, r2); fine_packed(b3, r3);
+            } else {
+                fine_wide(b0, r0 >> 1); fine_wide(b1, r1 >> 1); fine_wide(b2, r2 >> 1); fine_wide(b3, r3 >> 1);
+            }
         } else {
-            any(b0); any(b1); any(b2); any(b3);
+            any<PACKED>(b0); any<PACKED>(b1); any<PACKED>(b2); any<PACKED>(b3);
         }
     }
 };
 
-template <bool MAG>
+// Round 1 over grad[pb, pe): per element min / max and the cell histogram (count, sum of the low key
+// bits).  The bulk goes through packed cells (one shared-memory add per element instead of two, see
+// Round1Body::fine), folded into the wide counters every kPackTrips loop trips; the sum of the folded
+// counts is checked against the number of values that went in, and a mismatch (a cell took 256 values
+// or more within the trips: heavily repeated values) redoes those trips with the two-add path.
+// packed: kPackedCells zeroed words of shared memory, zero again on return.
+template <bool MAG, bool CLIP>
 __device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64_t pb, int64_t pe, int lo_e,
-                                              uint32_t* hist, float& vmin, float& vmax, uint32_t& nonfinite,
-                                              float tau)
+                                              uint32_t* hist, uint32_t* packed, float& vmin, float& vmax,
+                                              uint32_t& nonfinite, float tau)
 {
-    Round1Body<MAG> f;
+    __shared__ uint32_t sh_coarse, sh_total;
+    Round1Body<MAG, CLIP> f;
     f.tau = tau;
     f.lo23 = (uint32_t)lo_e << 23;
+    f.neg_lo23x2 = 0u - (f.lo23 << 1);
+    f.one24 = 0x01000000u;
     f.lo_e = lo_e;
     f.cnt = (uint32_t)__cvta_generic_to_shared(hist + (MAG ? 0 : kRound1Mag));
+    f.pk = (uint32_t)__cvta_generic_to_shared(packed);
+    f.coarse = (uint32_t)__cvta_generic_to_shared(&sh_coarse);
     f.mn = vmin; f.mx = vmax; f.nonfinite = nonfinite;
     int64_t a = (pb + 3) & ~(int64_t)3;
     if (a > pe) a = pe;
@@ -450,19 +500,74 @@ __device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64
     if (tid < (int)(a - pb)) f.one(__ldg(grad + pb + tid));
     if (tid < (int)(pe - b)) f.one(__ldg(grad + b + tid));
     const float4* g4 = reinterpret_cast<const float4*>(grad);
-    int64_t i = (a >> 2) + tid;
-    const int64_t e = b >> 2;
-    int64_t pf = (a >> 2) + (int64_t)kPrefetchTrips * 4 * kSelThreads;
-    for (; i + 3 * kSelThreads < e; i += 4 * kSelThreads) {
-        if (tid == 0 && pf + 4 * kSelThreads <= e) prefetch_l2(g4 + pf, kTripBytes);
-        pf += 4 * kSelThreads;
-        float4 x[4];
+    const int64_t first = a >> 2, e = b >> 2;
+    const int64_t ntrips = (e - first) / (4 * kSelThreads);  // full trips: the same for every thread
+    int64_t pf = first + (int64_t)kPrefetchTrips * 4 * kSelThreads;
+    constexpr int kNp = MAG ? kPackedPerSign : kPackedCells;
+    for (int64_t t0 = 0; t0 < ntrips; t0 += kPackTrips) {
+        const int nt = (int)((ntrips - t0 < kPackTrips) ? ntrips - t0 : kPackTrips);
+        if (tid == 0) { sh_coarse = 0u; sh_total = 0u; }
+        __syncthreads();
+        for (int tt = 0; tt < nt; ++tt) {
+            const int64_t i = first + (t0 + tt) * 4 * kSelThreads + tid;
+            if (tid == 0 && pf + 4 * kSelThreads <= e) prefetch_l2(g4 + pf, kTripBytes);
+            pf += 4 * kSelThreads;
+            float4 x[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i + u * kSelThreads);
+            for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i + u * kSelThreads);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) f.four(x[u]);
+            for (int u = 0; u < 4; ++u) f.template four<true>(x[u]);
+        }
+        __syncthreads();
+        // fold, phase 1: do the packed counts add up to the values that went in?
+        uint32_t mine = 0u;
+        for (int p = tid; p < kNp; p += kSelThreads) mine += packed[p] >> 24;
+        mine = __reduce_add_sync(0xffffffffu, mine);
+        if ((tid & 31) == 0 && mine) atomicAdd(&sh_total, mine);
+        __syncthreads();
+        const bool ok = sh_total + sh_coarse == (uint32_t)nt * 16u * kSelThreads;
+        // phase 2: into the wide counters (packed index p: negative values mirror below the middle)
+        for (int p = tid; p < kNp; p += kSelThreads) {
+            const uint32_t w = packed[p];
+            if (w) {
+                packed[p] = 0u;
+                if (ok) {
+                    // non-negative half: cell and low bits ascend with the magnitude; negative half: mirrored
+                    const uint32_t c = w >> 24, sum = w & 0xffffffu;
+                    const bool neg = !MAG && p >= kPackedPerSign;
+                    const int cell = MAG ? lo_e + p
+                                         : (neg ? kRound1Mag - 1 - lo_e - (p - kPackedPerSign) : kRound1Mag + lo_e + p);
+                    hist[cell] += c;
+                    const uint32_t add = neg ? c * ((1u << (23 - kSelM)) - 1u) - sum : sum;
+                    const uint32_t old = hist[kCells + cell];
+                    hist[kCells + cell] = old + add;
+                    if (old + add < old) hist[2 * kCells + cell] += 1u;  // carry into the high word
+                }
+            }
+        }
+        if (!ok) {
+            // a packed count wrapped: the fine values of these trips again, two adds each (the values outside
+            // the window were counted directly the first time and are skipped now)
+            __syncthreads();
+            for (int tt = 0; tt < nt; ++tt) {
+                const int64_t i = first + (t0 + tt) * 4 * kSelThreads + tid;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float4 x = __ldg(g4 + i + u * kSelThreads);
+                    const float vv[4] = {f.canon(x.x), f.canon(x.y), f.canon(x.z), f.canon(x.w)};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t bits = __float_as_uint(vv[j]);
+                        const uint32_t rel = (bits & 0x7fffffffu) - f.lo23;
+                        if (rel < ((uint32_t)kSelW << 23)) f.fine_wide(bits, rel);
+                    }
+                }
+            }
+        }
+        __syncthreads();  // everyone has read the totals before they are reset
     }
-    for (; i < e; i += kSelThreads) f.four(__ldg(g4 + i));
+    __syncthreads();
+    for (int64_t i = first + ntrips * 4 * kSelThreads + tid; i < e; i += kSelThreads) f.template four<false>(__ldg(g4 + i));
     vmin = f.mn; vmax = f.mx; nonfinite = f.nonfinite;
 }
 
@@ -1473,6 +1578,7 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         st->compact_only = compact_only ? 1 : 0;
         st->round = round + 1;
         st->arrive = 0;
+        st->arrived = 0ull;
         const int next = round + 1;
         st->cursor[next & 1] = 0ull;  // buffer the next round writes
         if (next == 3 && enqueue) {
@@ -1747,55 +1853,45 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         return hi_e;
     };
 
-    // Round 1 over one piece [pb_, pe_) of tensor t: histogram, min / max, arrival.  `alone`: the piece
-    // is the whole tensor.  Returns true when this CTA is the last one of the tensor to arrive; that
-    // CTA then runs r1_solve.
-    auto r1_stream = [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_, bool alone) -> bool {
-        const int64_t n = tend - tbeg;
-        TState* st = A.ws.st + t;
-        const int hi_e = window_anchor(tbeg, n);
-        const int lo_e = hi_e - kSelW;
-        const float tau = A.tau ? __ldg(A.tau + t) : __int_as_float(0x7f800000);
-        const int ncells = pb ? kRound1Mag : kRound1Cells;
-        uint32_t* gcnt = A.ws.gcnt + (size_t)t * kCells;
-        unsigned long long* glsum = A.ws.glsum + (size_t)t * kCells;
-        float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
-        uint32_t nf = 0u;
-        zero_hist(hist, ncells);
+    // Round 1 of a tensor on this CTA, in three steps: r1_begin clears the CTA's cells, r1_add streams
+    // a piece of the tensor into them (any number of pieces), r1_flush adds the cells to the tensor's
+    // global ones, reports `elems` streamed elements and returns true when that completes the tensor;
+    // the CTA for which it does runs r1_solve.
+    float r1_vmin = 0.f, r1_vmax = 0.f, r1_tau = 0.f;
+    uint32_t r1_nf = 0u;
+    int r1_lo_e = 0;
+    uint32_t* packed_cells = reinterpret_cast<uint32_t*>(smem + kSmemHist);
+    const int r1_ncells = pb ? kRound1Mag : kRound1Cells;
+    auto r1_begin = [&](int t, int64_t tbeg, int64_t tend) {
+        r1_lo_e = window_anchor(tbeg, tend - tbeg) - kSelW;
+        r1_tau = A.tau ? __ldg(A.tau + t) : 0.f;
+        r1_vmin = __int_as_float(0x7f800000);
+        r1_vmax = __int_as_float(0xff800000);
+        r1_nf = 0u;
         __syncthreads();
-        if (pb) stream_round1<true>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf, tau);
-        else stream_round1<false>(A.grad, pb_, pe_, lo_e, hist, vmin, vmax, nf, tau);
+        zero_hist(hist, r1_ncells);
+        for (int i = threadIdx.x; i < kPackedCells; i += kSelThreads) packed_cells[i] = 0u;
         __syncthreads();
-        // The low sums of the window's cells are 32 bits wide without a carry: exact as long as no such
-        // cell took more than 2^16 values.  Otherwise (heavily repeated values) the piece is redone in
-        // parts of kR1MaxPiece elements, flushed one by one.
-        bool crowded = false;
-        if (pe_ - pb_ > kR1MaxPiece) {
-            const int base = pb ? 0 : kRound1Mag;
-            for (int i = threadIdx.x; i < ncells; i += kSelThreads) {
-                const int mi = (i >= base) ? i - base : base - 1 - i;
-                crowded |= hist[i] > (uint32_t)kR1MaxPiece && mi >= lo_e && mi < lo_e + (kSelW << kSelM);
-            }
-        }
-        if (__syncthreads_or(crowded)) {
-            for (int64_t q = pb_; q < pe_; q += kR1MaxPiece) {
-                const int64_t qe = (q + kR1MaxPiece < pe_) ? q + kR1MaxPiece : pe_;
-                zero_hist(hist, ncells);
-                __syncthreads();
-                if (pb) stream_round1<true>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf, tau);
-                else stream_round1<false>(A.grad, q, qe, lo_e, hist, vmin, vmax, nf, tau);
-                __syncthreads();
-                flush_hist(hist, ncells, gcnt, glsum);
-                __syncthreads();
-            }
+    };
+    auto r1_add = [&](int64_t pb_, int64_t pe_) {
+        const bool clip = A.tau != nullptr;
+        if (pb) {
+            if (clip) stream_round1<true, true>(A.grad, pb_, pe_, r1_lo_e, hist, packed_cells, r1_vmin, r1_vmax, r1_nf, r1_tau);
+            else stream_round1<true, false>(A.grad, pb_, pe_, r1_lo_e, hist, packed_cells, r1_vmin, r1_vmax, r1_nf, r1_tau);
         } else {
-            flush_hist(hist, ncells, gcnt, glsum);
+            if (clip) stream_round1<false, true>(A.grad, pb_, pe_, r1_lo_e, hist, packed_cells, r1_vmin, r1_vmax, r1_nf, r1_tau);
+            else stream_round1<false, false>(A.grad, pb_, pe_, r1_lo_e, hist, packed_cells, r1_vmin, r1_vmax, r1_nf, r1_tau);
         }
+    };
+    auto r1_flush = [&](int t, int64_t n, int64_t elems) -> bool {
+        TState* st = A.ws.st + t;
+        __syncthreads();
+        flush_hist(hist, r1_ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         // min / max / non-finite: one atomic per warp
         {
-            const uint32_t kmin = __reduce_min_sync(0xffffffffu, float_to_key(vmin));  // +Inf / -Inf when the
-            const uint32_t kmax = __reduce_max_sync(0xffffffffu, float_to_key(vmax));  // thread saw nothing
-            const bool anynf = __any_sync(0xffffffffu, nf != 0u);
+            const uint32_t kmin = __reduce_min_sync(0xffffffffu, float_to_key(r1_vmin));  // +Inf / -Inf when the
+            const uint32_t kmax = __reduce_max_sync(0xffffffffu, float_to_key(r1_vmax));  // thread saw nothing
+            const bool anynf = __any_sync(0xffffffffu, r1_nf != 0u);
             if ((threadIdx.x & 31) == 0) {
                 atomicMax(&st->kmin_inv, ~kmin);
                 atomicMax(&st->kmax, kmax);
@@ -1804,16 +1900,13 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         }
         __threadfence();
         __syncthreads();
-        if (!alone) {
-            const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
-            if (threadIdx.x == 0) {
-                const unsigned prev = atomicAdd(&st->arrive, 1u);
-                sh_last = (prev == (unsigned)(c1 - c0));
-            }
-            __syncthreads();
-            if (!sh_last) return false;
-            __threadfence();
+        if (threadIdx.x == 0) {
+            const unsigned long long prev = atomicAdd(&st->arrived, (unsigned long long)elems);
+            sh_last = (prev + (unsigned long long)elems == (unsigned long long)n);
         }
+        __syncthreads();
+        if (!sh_last) return false;
+        __threadfence();
         return true;
     };
 
@@ -1870,32 +1963,56 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
                          A.tau ? __ldg(A.tau + t) : __int_as_float(0x7f800000));
         } else if (n <= kMidN) {
             // round 1 and its solver pass on this CTA; the tensor's CTA of the round-2 kernel goes on from there
-            r1_stream(t, tbeg, tend, tbeg, tend, true);
+            r1_begin(t, tbeg, tend);
+            r1_add(tbeg, tend);
+            r1_flush(t, n, n);
             r1_solve(t, tbeg, tend, true);
         }
         }();
         return;
     }
 
-    const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
-    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
-    // A CTA first streams all of its pieces and only then runs the solver passes of the tensors it
-    // finished, so that a solver pass never holds up the arrival of another tensor's piece.
+    // Flat CTAs: one chunk of the bucket each.  The solver passes of the tensors this CTA completed wait
+    // until its chunk has been streamed, so that a solver pass never holds up another tensor's arrival.
+    // (Handing smaller chunks out from a counter was tried and lost: the CTAs of a launch already finish
+    // within a few percent of one another, what ends late are the solver passes, and every extra chunk
+    // boundary costs a set-up and, in round 2, a drain of the compaction stages.)
     constexpr int kDefer = 8;
     int dt[kDefer];
     int nd = 0;
-    for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
-        if (tend - tbeg <= kMidN) return;
-        if (!r1_stream(t, tbeg, tend, pb_, pe_, false)) return;
-        if (nd < kDefer) {
+    int cur_t = -1;
+    int64_t cur_n = 0, cur_elems = 0;
+    auto done_with_current = [&]() {
+        if (cur_t < 0) return;
+        if (r1_flush(cur_t, cur_n, cur_elems)) {
+            if (nd < kDefer) {
 #pragma unroll
-            for (int u = 0; u < kDefer; ++u)
-                if (u == nd) dt[u] = t;
-            ++nd;
-        } else {
-            r1_solve(t, tbeg, tend, false);
+                for (int u = 0; u < kDefer; ++u)
+                    if (u == nd) dt[u] = cur_t;
+                ++nd;
+            } else {
+                r1_solve(cur_t, __ldg(A.off + cur_t), __ldg(A.off + cur_t + 1), false);
+            }
         }
-    });
+        cur_t = -1;
+    };
+    {
+        const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
+        const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+        for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+            if (tend - tbeg <= kMidN) return;
+            if (t != cur_t) {
+                done_with_current();
+                r1_begin(t, tbeg, tend);
+                cur_t = t;
+                cur_n = tend - tbeg;
+                cur_elems = 0;
+            }
+            r1_add(pb_, pe_);
+            cur_elems += pe_ - pb_;
+        });
+    }
+    done_with_current();
 #pragma unroll
     for (int u = 0; u < kDefer; ++u)
         if (u < nd) r1_solve(dt[u], __ldg(A.off + dt[u]), __ldg(A.off + dt[u] + 1), false);
@@ -1910,26 +2027,34 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
     const bool pb = A.scheme == OGQ_BINGRAD_PB;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
 
-    // Second pass over the piece [pb_, pe_) of tensor t: copies the values inside the tensor's
-    // intervals (and counts them on the finer cells unless they already fit one sort).
-    auto r2_stream = [&](int t, int64_t tbeg, int64_t pb_, int64_t pe_, bool& copy_only) {
+    // Second pass over a tensor on this CTA, in three steps like round 1: r2_begin builds the tensor's
+    // interval table and prefilter and clears the CTA's cells, r2_add streams a piece (copies the values
+    // inside the intervals and counts them on the finer cells, unless they already fit one sort),
+    // r2_flush adds the cells to the tensor's global ones.
+    bool r2_copy_only = false;
+    auto r2_begin = [&](int t) {
         TState* st = A.ws.st + t;
         __syncthreads();
         table_from_intervals_cta(tb, st->iv, __ldcg(&st->m));
         __syncthreads();
         build_prefilter(tb, pb);
-        copy_only = __ldcg(&st->compact_only) != 0;
-        if (!copy_only) zero_hist(hist, tb.ncells);
+        r2_copy_only = __ldcg(&st->compact_only) != 0;
+        if (!r2_copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
+    };
+    auto r2_add = [&](int t, int64_t tbeg, int64_t pb_, int64_t pe_) {
+        TState* st = A.ws.st + t;
         uint32_t* stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
         if (A.tau)
             stream_round2<true>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stage,
-                                A.ws.buf[0] + tbeg, &st->cursor[0], copy_only, __ldg(A.tau + t));
+                                A.ws.buf[0] + tbeg, &st->cursor[0], r2_copy_only, __ldg(A.tau + t));
         else
             stream_round2<false>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stage,
-                                 A.ws.buf[0] + tbeg, &st->cursor[0], copy_only, 0.f);
+                                 A.ws.buf[0] + tbeg, &st->cursor[0], r2_copy_only, 0.f);
+    };
+    auto r2_flush = [&](int t) {
         __syncthreads();
-        if (!copy_only) flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
+        if (!r2_copy_only) flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         __threadfence();
         __syncthreads();
     };
@@ -1942,9 +2067,10 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
         const int64_t n = tend - tbeg;
         TState* st = A.ws.st + t;
         if (n <= kSmallN || n > kMidN || __ldcg(&st->done)) return;
-        bool copy_only;
-        r2_stream(t, tbeg, tbeg, tend, copy_only);
-        if (copy_only) {
+        r2_begin(t);
+        r2_add(t, tbeg, tbeg, tend);
+        r2_flush(t);
+        if (r2_copy_only) {
             finish_sorted(st, t, A.s, A.ws.buf[0] + tbeg, A.levels, A.status, smem, S, 0);
             return;
         }
@@ -1955,10 +2081,7 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
         return;
     }
 
-    const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
-    const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
-    // as in round 1, the solver passes of the tensors this CTA finished wait until all of its pieces
-    // have been streamed
+    // flat CTAs: one chunk each, solver passes last (as in round 1)
     constexpr int kDefer = 8;
     int dt[kDefer];
     int nd = 0;
@@ -1972,30 +2095,49 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
         solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
                      A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, true, smem, S);
     };
-    for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
-        const int64_t n = tend - tbeg;
-        if (n <= kMidN) return;
-        TState* st = A.ws.st + t;
-        if (__ldcg(&st->done)) return;
-        bool copy_only;
-        r2_stream(t, tbeg, pb_, pe_, copy_only);
-        const int64_t c0 = tbeg / A.chunk, c1 = (tend - 1) / A.chunk;
+    int cur_t = -1;
+    int64_t cur_n = 0, cur_elems = 0;
+    auto done_with_current = [&]() {
+        if (cur_t < 0) return;
+        r2_flush(cur_t);
+        TState* st = A.ws.st + cur_t;
         if (threadIdx.x == 0) {
-            const unsigned prev = atomicAdd(&st->arrive, 1u);
-            sh_last = (prev == (unsigned)(c1 - c0));
+            const unsigned long long prev = atomicAdd(&st->arrived, (unsigned long long)cur_elems);
+            sh_last = (prev + (unsigned long long)cur_elems == (unsigned long long)cur_n);
         }
         __syncthreads();
-        if (!sh_last) return;
-        __threadfence();
-        if (nd < kDefer) {
+        if (sh_last) {
+            __threadfence();
+            if (nd < kDefer) {
 #pragma unroll
-            for (int u = 0; u < kDefer; ++u)
-                if (u == nd) dt[u] = t;
-            ++nd;
-        } else {
-            finish(t);
+                for (int u = 0; u < kDefer; ++u)
+                    if (u == nd) dt[u] = cur_t;
+                ++nd;
+            } else {
+                finish(cur_t);
+            }
         }
-    });
+        cur_t = -1;
+    };
+    {
+        const int64_t lo = (int64_t)(blockIdx.x - A.T) * A.chunk;
+        const int64_t hi = (lo + A.chunk < A.total) ? lo + A.chunk : A.total;
+        for_each_piece(A.off, A.T, lo, hi, [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+            const int64_t n = tend - tbeg;
+            if (n <= kMidN) return;
+            if (t != cur_t) {
+                done_with_current();
+                if (__ldcg(&A.ws.st[t].done)) return;  // settled in round 1
+                r2_begin(t);
+                cur_t = t;
+                cur_n = n;
+                cur_elems = 0;
+            }
+            r2_add(t, tbeg, pb_, pe_);
+            cur_elems += pe_ - pb_;
+        });
+    }
+    done_with_current();
 #pragma unroll
     for (int u = 0; u < kDefer; ++u)
         if (u < nd) finish(dt[u]);
