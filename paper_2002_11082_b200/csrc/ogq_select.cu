@@ -51,6 +51,8 @@ struct TState {
     unsigned long long arrived;  // elements of the current pass whose counts have been flushed
     unsigned expected;
     int compact_only;  // the next pass only copies the keys inside the intervals: they fit one sort
+    int overflow;      // the current pass dropped copies that did not fit the tensor's region
+    int from_grad;     // the current pass (round >= 3) reads the gradient, not the previous pass's copies
     unsigned long long cursor[2];
     long long n;
     double stot;
@@ -64,8 +66,16 @@ struct SelWs {
     unsigned long long* glsum;   // [T][kCells]
     unsigned* nitems;            // [1] work items of round 3
     int2* items;                 // [T * kMaxSlices]
-    uint32_t* buf[2];            // [total] copied keys, tensor t at its element offset
+    uint32_t* buf[2];            // [total / kBufDiv] copied keys: tensor t owns [sel_region(off[t]), sel_region(off[t+1]))
 };
+
+// The copied keys of a tensor are normally a few percent of it, so the two key buffers hold one eighth
+// of the bucket: the tensor that starts at element x owns the words from sel_region(x) on, up to where
+// the next tensor's region starts.  A pass whose copies do not fit drops the surplus and marks the
+// tensor (TState::overflow); the next pass then reads the gradient again instead of the buffer, with
+// narrower intervals, until the copies fit.
+constexpr int kBufDiv = 8;
+__host__ __device__ __forceinline__ int64_t sel_region(int64_t x) { return (x / kBufDiv) & ~(int64_t)3; }
 
 static size_t sel_zero_bytes(int T)
 {
@@ -76,7 +86,7 @@ static size_t sel_zero_bytes(int T)
 size_t ws_bytes_select(int T, int64_t total, int /*s*/)
 {
     return sel_zero_bytes(T) + align_up(sizeof(int2) * (size_t)T * kMaxSlices, 256) +
-           2 * align_up(sizeof(uint32_t) * (size_t)(total + 4), 256);
+           2 * align_up(sizeof(uint32_t) * (size_t)(total / kBufDiv + 8), 256);
 }
 
 static SelWs sel_carve(void* base, int T, int64_t total)
@@ -88,7 +98,7 @@ static SelWs sel_carve(void* base, int T, int64_t total)
     w.glsum = (unsigned long long*)p; p += align_up(sizeof(unsigned long long) * (size_t)T * kCells, 256);
     w.nitems = (unsigned*)p; p += 256;
     w.items = (int2*)p; p += align_up(sizeof(int2) * (size_t)T * kMaxSlices, 256);
-    w.buf[0] = (uint32_t*)p; p += align_up(sizeof(uint32_t) * (size_t)(total + 4), 256);
+    w.buf[0] = (uint32_t*)p; p += align_up(sizeof(uint32_t) * (size_t)(total / kBufDiv + 8), 256);
     w.buf[1] = (uint32_t*)p;
     return w;
 }
@@ -582,6 +592,8 @@ struct Round2Ctx {  // per-CTA constants of round 2, kept in shared memory to sp
     unsigned long long* cursor;
     uint32_t clear;  // 0x7fffffff when only magnitudes count
     int nohist;      // copy the keys inside the intervals without counting them
+    unsigned long long cap;  // words of the tensor's region in the destination buffer
+    int* overflow;           // set when a copy did not fit
 };
 
 // Phase B of round 2 for one warp: classifies `fill` parked values 32 at a time.  A free function
@@ -610,7 +622,11 @@ __device__ __noinline__ void round2_drain(const Table* tb, const Round2Ctx* ctx,
             unsigned long long pos = 0;
             if (lane == 0) pos = atomicAdd(ctx->cursor, (unsigned long long)__popc(m2));
             pos = __shfl_sync(0xffffffffu, pos, 0);
-            if (in) ctx->dst[pos + __popc(m2 & lt)] = key;
+            if (in) {
+                const unsigned long long at = pos + __popc(m2 & lt);
+                if (at < ctx->cap) ctx->dst[at] = key;
+                else *(volatile int*)ctx->overflow = 1;
+            }
         }
     }
     __syncwarp();
@@ -688,8 +704,8 @@ struct Round2Warp {
 template <bool CLIP>
 __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64_t pb, int64_t pe,
                                               bool magnitude_only, const Table& tb, uint32_t* cnt, uint32_t* lo,
-                                              uint32_t* hi, uint32_t* stage, uint32_t* dst,
-                                              unsigned long long* cursor, bool nohist, float tau)
+                                              uint32_t* hi, uint32_t* stage, uint32_t* dst, int64_t cap,
+                                              unsigned long long* cursor, int* overflow, bool nohist, float tau)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __shared__ Round2Ctx ctx;
@@ -699,6 +715,8 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
         ctx.cnt = cnt; ctx.lo = lo; ctx.hi = hi; ctx.dst = dst; ctx.cursor = cursor;
         ctx.clear = magnitude_only ? 0x7fffffffu : 0xffffffffu;
         ctx.nohist = nohist ? 1 : 0;
+        ctx.cap = (unsigned long long)cap;
+        ctx.overflow = overflow;
     }
     if (lane == 0) fills[warp] = 0;
     __syncthreads();
@@ -1310,7 +1328,7 @@ __device__ bool refine_parallel(SolverShared& S, bool trim_empty)
 __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long long* glsum, int scheme,
                              int s, float* __restrict__ levels, int32_t* __restrict__ status,
                              unsigned* nitems, int2* items, const uint32_t* round_buf, bool enqueue,
-                             unsigned char* smem, SolverShared& S)
+                             unsigned char* smem, SolverShared& S, int64_t cap)
 {
     constexpr size_t kOffSpre = (kSlots * sizeof(uint32_t) + 15) / 16 * 16;
     uint32_t* cpre = reinterpret_cast<uint32_t*>(smem);
@@ -1555,7 +1573,9 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
         if (threadIdx.x == 0) { st->done = 1; __threadfence(); }
         return true;
     }
-    if (!pb && round >= 2 && S.cand <= kSmallN && round_buf != nullptr) {
+    // (the copies of the pass that just ended are complete unless it overflowed its region)
+    const bool incomplete = round >= 2 && __ldcg(&st->overflow) != 0;
+    if (!pb && round >= 2 && S.cand <= kSmallN && round_buf != nullptr && !incomplete) {
         const long long src_cnt = (long long)__ldcg(&st->cursor[round & 1]);
         if (src_cnt <= kSortScanMax) {
             sort_finish(st, t, s, round_buf, src_cnt, levels, status, smem, S);
@@ -1565,7 +1585,7 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     // prepare the next round: clear the cells it will use, publish the new intervals.  When the
     // elements inside the new intervals already fit one sort (ORQ), the next pass only copies them
     // and its last CTA sorts and finishes the tensor (finish_sorted): no cells, no further solver pass.
-    const bool compact_only = !pb && S.cand <= kSmallN;
+    const bool compact_only = !pb && S.cand <= kSmallN && S.cand <= cap;
     const int ncells_next = S.niv[S.nm - 1].cellbase + S.niv[S.nm - 1].ncell;
     if (!compact_only)
         for (int i = threadIdx.x; i < ncells_next; i += kSelThreads) {
@@ -1576,13 +1596,17 @@ __device__ bool solver_round(TState* st, int t, uint32_t* gcnt, unsigned long lo
     if (threadIdx.x == 0) {
         st->m = S.nm;
         st->compact_only = compact_only ? 1 : 0;
+        st->from_grad = incomplete ? 1 : 0;  // the next pass cannot read copies that were cut short
+        st->overflow = 0;
         st->round = round + 1;
         st->arrive = 0;
         st->arrived = 0ull;
         const int next = round + 1;
         st->cursor[next & 1] = 0ull;  // buffer the next round writes
         if (next == 3 && enqueue) {
-            const unsigned long long cntk = __ldcg(&st->cursor[0]);
+            // work items of the round-3 kernel: slices of the copied keys, or of the tensor itself when
+            // the copies were cut short
+            const unsigned long long cntk = incomplete ? (unsigned long long)(st->n / 16) : __ldcg(&st->cursor[0]);
             unsigned ns = (unsigned)((cntk + kSliceElems - 1) / kSliceElems);
             if (ns < 1) ns = 1;
             if (ns > kMaxSlices) ns = kMaxSlices;
@@ -1773,6 +1797,25 @@ struct SelArgs {
     SelWs ws;
 };
 
+// One pass over grad[pb_, pe_) of tensor t with the tensor's current intervals (table and prefilter
+// already built in tb): the values inside the intervals are copied to key buffer k (what fits the
+// tensor's region) and, unless copy_only, counted on the cells.
+__device__ __forceinline__ void grad_pass(const SelArgs& A, int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_,
+                                          int k, const Table& tb, uint32_t* hist, unsigned char* smem, bool copy_only)
+{
+    TState* st = A.ws.st + t;
+    uint32_t* stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+    uint32_t* dst = A.ws.buf[k] + sel_region(tbeg);
+    const int64_t cap = sel_region(tend) - sel_region(tbeg);
+    const bool mag = A.scheme == OGQ_BINGRAD_PB;
+    if (A.tau)
+        stream_round2<true>(A.grad, pb_, pe_, mag, tb, hist, hist + kCells, hist + 2 * kCells, stage, dst, cap,
+                            &st->cursor[k], &st->overflow, copy_only, __ldg(A.tau + t));
+    else
+        stream_round2<false>(A.grad, pb_, pe_, mag, tb, hist, hist + kCells, hist + 2 * kCells, stage, dst, cap,
+                             &st->cursor[k], &st->overflow, copy_only, 0.f);
+}
+
 // Continues the rounds of one tensor on a single CTA until it is finished (the working set is
 // tiny by then).  Called by the CTA that completed round >= 3.
 __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table& tb, SolverShared& S)
@@ -1781,7 +1824,7 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
     uint32_t* gcnt = A.ws.gcnt + (size_t)t * kCells;
     unsigned long long* glsum = A.ws.glsum + (size_t)t * kCells;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem);
-    const int64_t tbeg = __ldg(A.off + t);
+    const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
     for (int guard = 0; guard < kMaxRounds; ++guard) {
         const int round = st->round;
         const uint32_t* src = A.ws.buf[(round - 1) & 1];  // 16-byte aligned base; indices are absolute
@@ -1792,27 +1835,33 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
         __syncthreads();
         if (!copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
-        Stager stg;
-        stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
-        stg.dst = A.ws.buf[round & 1] + tbeg;
-        stg.cursor = &st->cursor[round & 1];
-        stg.fill = 0;
-        uint32_t kmin = 0, kmax = 0, nf = 0;
-        stream_piece<false, false, true>(src, tbeg, tbeg + cnt, false, tb, hist, hist + kCells, hist + 2 * kCells,
-                                         stg, kmin, kmax, nf, copy_only);
-        stg.flush();
+        if (st->from_grad) {
+            // the previous pass's copies did not fit: this pass reads the tensor itself again
+            build_prefilter(tb, A.scheme == OGQ_BINGRAD_PB);
+            grad_pass(A, t, tbeg, tend, tbeg, tend, round & 1, tb, hist, smem, copy_only);
+        } else {
+            Stager stg;
+            stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+            stg.dst = A.ws.buf[round & 1] + sel_region(tbeg);
+            stg.cursor = &st->cursor[round & 1];
+            stg.fill = 0;
+            uint32_t kmin = 0, kmax = 0, nf = 0;
+            stream_piece<false, false, true>(src, sel_region(tbeg), sel_region(tbeg) + cnt, false, tb, hist, hist + kCells,
+                                             hist + 2 * kCells, stg, kmin, kmax, nf, copy_only);
+            stg.flush();
+        }
         __syncthreads();
         if (copy_only) {
             __threadfence();
             __syncthreads();
-            finish_sorted(st, t, A.s, A.ws.buf[round & 1] + tbeg, A.levels, A.status, smem, S, round & 1);
+            finish_sorted(st, t, A.s, A.ws.buf[round & 1] + sel_region(tbeg), A.levels, A.status, smem, S, round & 1);
             return;
         }
         flush_hist(hist, tb.ncells, gcnt, glsum);
         __threadfence();
         __syncthreads();
         if (solver_round(st, t, gcnt, glsum, A.scheme, A.s, A.levels, A.status, A.ws.nitems, A.ws.items,
-                         A.ws.buf[round & 1] + tbeg, false, smem, S))
+                         A.ws.buf[round & 1] + sel_region(tbeg), false, smem, S, sel_region(tend) - sel_region(tbeg)))
             return;
     }
     if (threadIdx.x == 0) {
@@ -1944,7 +1993,7 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArg
         bool done;
         done = solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells,
                                            A.scheme, A.s, A.levels, A.status, A.ws.nitems, A.ws.items, nullptr,
-                                           !alone, smem, S);
+                                           !alone, smem, S, sel_region(tend) - sel_region(tbeg));
         return done;
     };
 
@@ -2042,15 +2091,8 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
         if (!r2_copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
     };
-    auto r2_add = [&](int t, int64_t tbeg, int64_t pb_, int64_t pe_) {
-        TState* st = A.ws.st + t;
-        uint32_t* stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
-        if (A.tau)
-            stream_round2<true>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stage,
-                                A.ws.buf[0] + tbeg, &st->cursor[0], r2_copy_only, __ldg(A.tau + t));
-        else
-            stream_round2<false>(A.grad, pb_, pe_, pb, tb, hist, hist + kCells, hist + 2 * kCells, stage,
-                                 A.ws.buf[0] + tbeg, &st->cursor[0], r2_copy_only, 0.f);
+    auto r2_add = [&](int t, int64_t tbeg, int64_t tend, int64_t pb_, int64_t pe_) {
+        grad_pass(A, t, tbeg, tend, pb_, pe_, 0, tb, hist, smem, r2_copy_only);
     };
     auto r2_flush = [&](int t) {
         __syncthreads();
@@ -2068,14 +2110,14 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
         TState* st = A.ws.st + t;
         if (n <= kSmallN || n > kMidN || __ldcg(&st->done)) return;
         r2_begin(t);
-        r2_add(t, tbeg, tbeg, tend);
+        r2_add(t, tbeg, tend, tbeg, tend);
         r2_flush(t);
         if (r2_copy_only) {
-            finish_sorted(st, t, A.s, A.ws.buf[0] + tbeg, A.levels, A.status, smem, S, 0);
+            finish_sorted(st, t, A.s, A.ws.buf[0] + sel_region(tbeg), A.levels, A.status, smem, S, 0);
             return;
         }
         if (solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                         A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, false, smem, S))
+                         A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + sel_region(tbeg), false, smem, S, sel_region(tend) - sel_region(tbeg)))
             return;
         finish_alone(A, t, smem, tb, S);
         return;
@@ -2087,13 +2129,13 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
     int nd = 0;
     auto finish = [&](int t) {
         TState* st = A.ws.st + t;
-        const int64_t tbeg = __ldg(A.off + t);
+        const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
         if (__ldcg(&st->compact_only) != 0) {
-            finish_sorted(st, t, A.s, A.ws.buf[0] + tbeg, A.levels, A.status, smem, S, 0);
+            finish_sorted(st, t, A.s, A.ws.buf[0] + sel_region(tbeg), A.levels, A.status, smem, S, 0);
             return;
         }
         solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                     A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + tbeg, true, smem, S);
+                     A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[0] + sel_region(tbeg), true, smem, S, sel_region(tend) - sel_region(tbeg));
     };
     int cur_t = -1;
     int64_t cur_n = 0, cur_elems = 0;
@@ -2133,7 +2175,7 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round2(SelArg
                 cur_n = n;
                 cur_elems = 0;
             }
-            r2_add(t, tbeg, pb_, pe_);
+            r2_add(t, tbeg, tend, pb_, pe_);
             cur_elems += pe_ - pb_;
         });
     }
@@ -2156,9 +2198,10 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
         const int2 it = A.ws.items[w];
         const int t = it.x;
         TState* st = A.ws.st + t;
-        const int64_t tbeg = __ldg(A.off + t);
+        const int64_t tbeg = __ldg(A.off + t), tend = __ldg(A.off + t + 1);
         const unsigned ns = __ldcg(&st->expected);
-        const int64_t cnt = (int64_t)__ldcg(&st->cursor[0]);
+        const bool from_grad = __ldcg(&st->from_grad) != 0;  // round 2's copies were cut short: slices of the tensor
+        const int64_t cnt = from_grad ? tend - tbeg : (int64_t)__ldcg(&st->cursor[0]);
         int64_t per = (cnt + ns - 1) / ns;
         per = (per + 3) & ~(int64_t)3;
         int64_t pb_ = per * it.y, pe_ = pb_ + per;
@@ -2170,15 +2213,20 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
         __syncthreads();
         if (!copy_only) zero_hist(hist, tb.ncells);
         __syncthreads();
-        Stager stg;
-        stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
-        stg.dst = A.ws.buf[1] + tbeg;
-        stg.cursor = &st->cursor[1];
-        stg.fill = 0;
-        uint32_t kmin = 0, kmax = 0, nf = 0;
-        stream_piece<false, false, true>(A.ws.buf[0], tbeg + pb_, tbeg + pe_, false, tb, hist, hist + kCells,
-                                         hist + 2 * kCells, stg, kmin, kmax, nf, copy_only);
-        stg.flush();
+        if (from_grad) {
+            build_prefilter(tb, A.scheme == OGQ_BINGRAD_PB);
+            grad_pass(A, t, tbeg, tend, tbeg + pb_, tbeg + pe_, 1, tb, hist, smem, copy_only);
+        } else {
+            Stager stg;
+            stg.stage = reinterpret_cast<uint32_t*>(smem + kSmemHist) + (threadIdx.x >> 5) * kStageCap;
+            stg.dst = A.ws.buf[1] + sel_region(tbeg);
+            stg.cursor = &st->cursor[1];
+            stg.fill = 0;
+            uint32_t kmin = 0, kmax = 0, nf = 0;
+            stream_piece<false, false, true>(A.ws.buf[0], sel_region(tbeg) + pb_, sel_region(tbeg) + pe_, false, tb, hist,
+                                             hist + kCells, hist + 2 * kCells, stg, kmin, kmax, nf, copy_only);
+            stg.flush();
+        }
         __syncthreads();
         if (!copy_only) flush_hist(hist, tb.ncells, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells);
         __threadfence();
@@ -2191,11 +2239,11 @@ __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round3(SelArg
         if (!sh_last) continue;
         __threadfence();
         if (copy_only) {
-            finish_sorted(st, t, A.s, A.ws.buf[1] + tbeg, A.levels, A.status, smem, S, 1);
+            finish_sorted(st, t, A.s, A.ws.buf[1] + sel_region(tbeg), A.levels, A.status, smem, S, 1);
             continue;
         }
         if (!solver_round(st, t, A.ws.gcnt + (size_t)t * kCells, A.ws.glsum + (size_t)t * kCells, A.scheme, A.s,
-                          A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[1] + tbeg, false, smem, S))
+                          A.levels, A.status, A.ws.nitems, A.ws.items, A.ws.buf[1] + sel_region(tbeg), false, smem, S, sel_region(tend) - sel_region(tbeg)))
             finish_alone(A, t, smem, tb, S);
     }
 }

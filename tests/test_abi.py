@@ -65,3 +65,11 @@ def test_selection_solvers_refuse_buckets_of_2_to_the_32_elements():
         ogq.ogq_levels_bingrad(dummy, dummy, 1, big, ogq.OGQ_BINGRAD_PB, 0, dummy, dummy, dummy, dummy, 1 << 40,
                                stream=0)
     assert e.value.code == 2
+
+
+def test_workspace_of_the_vgg19_bucket_is_a_fraction_of_the_gradient():
+    """The key buffers hold one eighth of the bucket each (copies that do not fit make the solver read
+    the gradient again): 143.7 M elements need well under 0.3 GB of scratch."""
+    ws = ogq.ogq_workspace_bytes(38, 143667240, 17)
+    assert ws < 0.3e9
+    assert ws < 1.2 * 143667240 + 38 * 100_000
