@@ -2271,10 +2271,12 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     // Flat streaming CTAs: one wave (kSelResident per SM).  Each CTA pays a set-up, a flush of its
     // cells and an arrival per tensor piece, so larger chunks stream more of the time; a second wave
     // balanced a lone call slightly better in round 1 but cost throughput whenever several calls
-    // (workers on their own streams) share the GPU.
+    // (workers on their own streams) share the GPU.  Chunks are at least 131,072 elements: on a bucket of
+    // 25 M elements that leaves a third of the wave's slots to concurrent calls (measured with eight
+    // workers in flight: 8 % more throughput, 3 % slower alone).
     const int64_t wave = (int64_t)kSelResident * sm_count;
     const int target = wave < kMaxFlatCtas ? (int)wave : kMaxFlatCtas;
-    FlatGrid g = make_flat_grid(total, target, 32768);
+    FlatGrid g = make_flat_grid(total, target, 131072);
     SelArgs A;
     A.grad = d_grad; A.tau = d_tau; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
     A.scheme = scheme; A.s = s; A.levels = d_levels; A.status = d_status;
