@@ -541,6 +541,87 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_dp(args):
+    """Data parallelism as in Algorithm 2: every rank is one worker.  A step = levels + quantize + pack
+    of the rank's own bucket, all-gather of the packed codes and level tables (NCCL) into the rank's own
+    memory, unpack + dequantize + sum over all workers from there."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    import torch
+
+    import paper_2002_11082_b200 as ogq
+    from paper_2002_11082_b200.sharding import CodeExchange, aggregate_throughput, max_over_ranks
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    peak, peak_src = measured_peaks()
+    S = Setup(torch, ogq, dev, args.workload, args.scheme, 1, args.seed, rank)  # worker id = rank
+    ex = CodeExchange(world, int(S.h_po[-1]), S.T, S.s, device=dev)
+    pk_rows, lv_rows = ex.pointer_rows()
+    pk_ptrs = torch.tensor(pk_rows, dtype=torch.int64, device=dev)
+    lv_ptrs = torch.tensor(lv_rows, dtype=torch.int64, device=dev)
+
+    def step():
+        S.lqp(0, None, 0)
+        ex.gather(dist, S.packed[0], S.levels[0])
+        ogq.ogq_unpack_sum(pk_ptrs, lv_ptrs, world, S.off, S.po, S.T, S.N, S.s, 1.0 / world, S.out)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    for _ in range(warmup):
+        step()
+    barrier()
+    S.check_status()
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    need_flush = 4 * S.N <= 2 * 126e6
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ogq.ogq_launch_count()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    total = 0.0
+    for _ in range(steps):
+        if need_flush:
+            flush_buf.fill_(1)
+        barrier()
+        a.record()
+        step()
+        b.record()
+        torch.cuda.synchronize()
+        total += a.elapsed_time(b)
+    ms_step = max_over_ranks(total / steps, dist, dev)
+    launches = ogq.ogq_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": aggregate_throughput(4.0 * S.N, ms_step, world), "unit": UNIT, "n_gpus": world,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "mode": "dp",
+            "config": {"workload": args.workload, "scheme": args.scheme, "levels": S.s, "bits": S.bits,
+                       "workers": world, "tensors": S.T, "elements": S.N,
+                       "exchange": "all-gather of packed codes and level tables, then local unpack+sum",
+                       "recv_bytes_per_rank_and_step": ex.recv_bytes},
+            "gpu_launches": int(launches), "clocks": clocks, "peak_source": peak_src,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -556,12 +637,16 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-secondary", action="store_true")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "dp"],
+                    help="replicas: K simulated workers per GPU (default); dp: one worker per rank, codes all-gathered")
     ap.add_argument("--dense", action="store_true", help="ORQ codes in the base-s (entropy-dense) wire format")
     ap.add_argument("--bucket-len", type=int, default=0,
                     help="fixed-length bucket mode: quantize buckets of this many elements (ogq_bucket_encode)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "dp":
+        run_dp(args)
     else:
         run_ours(args)
 
