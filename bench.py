@@ -309,6 +309,10 @@ class Setup:
                                   self.thresh[k], self.seed, k, self.po, self.packed[k], stream)
 
     def unpack(self):
+        if self.bucket_len:
+            self.ogq.ogq_bucket_decode_sum(self.pk_ptrs, self.lv_ptrs, self.K, self.N, self.bucket_len, self.s,
+                                           1.0 / self.K, self.out)
+            return
         if self.dense:
             self.ogq.ogq_unpack_sum_dense(self.pk_ptrs, self.lv_ptrs, self.K, self.off, self.po, self.T, self.N, self.s,
                                           1.0 / self.K, self.out)
@@ -458,6 +462,7 @@ def run_ours(args):
         "k_sel_round1": 4.0 * N, "k_sel_round2": 4.0 * N, "k_sel_round3": 0.0, "k_bb_pass": 4.0 * N,
         "k_quantize_pack_random": (4.0 + bits / 8.0) * N, "k_quantize_pack_threshold": (4.0 + 1 / 8.0) * N,
         "k_unpack_sum": (K * bits / 8.0 + 4.0) * N, "k_bucket_encode": (4.0 + bits / 8.0) * N,
+        "k_bucket_decode_sum": (K * bits / 8.0 + 4.0) * N,
         "k_quantize_pack_dense": (4.0 + bits / 8.0) * N, "k_unpack_sum_dense": (K * bits / 8.0 + 4.0) * N,
     }
     kernels = {}

@@ -277,6 +277,16 @@ ogq_status ogq_bucket_encode(const float *d_grad, int64_t total_elems, int d, og
                              ogq_stream_t stream);
 
 /*
+ * Server step of Algorithm 2 for fixed-length buckets: out[i] = scale * sum_{k<K}
+ * levels_k[i / d][code_k[i]], fp32 sum in worker order, the result ogq_unpack_sum gives for
+ * offsets j d.  d_packed_k / d_levels_k: DEVICE arrays of K device pointers to the workers' packed
+ * buffers and [nb][s] level tables as ogq_bucket_encode wrote them.  1 <= K <= 64.  No scratch.
+ */
+ogq_status ogq_bucket_decode_sum(const uint32_t *const *d_packed_k, const float *const *d_levels_k, int K,
+                                 int64_t total_elems, int d, int s, float scale, float *d_out,
+                                 ogq_stream_t stream);
+
+/*
  * Measurement helpers (no counterpart in the paper; they do not touch the data path).
  * ogq_launch_count: number of kernels this library has launched in this process so far.
  * ogq_profile_enable(1): from now on every kernel launch of the library is bracketed by two CUDA

@@ -39,6 +39,7 @@ from .binding import (  # noqa: F401
     ogq_quantize_pack_clipped,
     ogq_bucket_packed_words,
     ogq_bucket_encode,
+    ogq_bucket_decode_sum,
     ogq_launch_count,
     ogq_profile_enable,
     ogq_profile_collect,

@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
                                                 vp, vp, vp]
         L.ogq_levels_bingrad_clipped.restype = i32
         L.ogq_levels_bingrad_clipped.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.ogq_bucket_decode_sum.restype = i32
+        L.ogq_bucket_decode_sum.argtypes = [vp, vp, i32, i64, i32, i32, ctypes.c_float, vp, vp]
         L.ogq_launch_count.restype = ctypes.c_ulonglong
         L.ogq_launch_count.argtypes = []
         L.ogq_profile_enable.restype = i32
@@ -289,6 +291,15 @@ def ogq_bucket_encode(d_grad, total_elems: int, d: int, scheme: int, s: int, ite
                                 int(seed) & 0xFFFFFFFFFFFFFFFF, int(stream_id) & 0xFFFFFFFF, _ptr(d_levels),
                                 _ptr(d_thresh), _ptr(d_status), _ptr(d_packed), _stream(stream)),
         "ogq_bucket_encode",
+    )
+
+
+def ogq_bucket_decode_sum(d_packed_k, d_levels_k, K: int, total_elems: int, d: int, s: int, scale: float, d_out,
+                          stream=None) -> None:
+    _check(
+        lib().ogq_bucket_decode_sum(_ptr(d_packed_k), _ptr(d_levels_k), int(K), int(total_elems), int(d), int(s),
+                                    float(scale), _ptr(d_out), _stream(stream)),
+        "ogq_bucket_decode_sum",
     )
 
 

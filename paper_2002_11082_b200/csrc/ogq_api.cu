@@ -60,7 +60,7 @@ bool select_size_ok(int64_t total_elems) { return total_elems < ((int64_t)1 << 3
 
 extern "C" {
 
-const char* ogq_version(void) { return "ogq 0.1 (sm_100a)"; }
+const char* ogq_version(void) { return "ogq 0.2 (sm_100a)"; }
 
 unsigned long long ogq_launch_count(void) { return ogq::g_launches.load(std::memory_order_relaxed); }
 
@@ -414,6 +414,22 @@ ogq_status ogq_bucket_encode(const float* d_grad, int64_t total_elems, int d, og
     if (sms <= 0) return OGQ_ERR_CUDA;
     cudaError_t e = ogq::launch_bucket_encode(d_grad, total_elems, d, (int)scheme, s, iters, clip_c, seed, stream_id,
                                               d_levels, d_thresh, d_status, d_packed, sms, (cudaStream_t)stream);
+    return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
+}
+
+ogq_status ogq_bucket_decode_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                                 int64_t total_elems, int d, int s, float scale, float* d_out, ogq_stream_t stream)
+{
+    if (total_elems < 0 || !d_packed_k || !d_levels_k) return OGQ_ERR_INVALID_ARG;
+    if (K < 1 || K > 64) return OGQ_ERR_INVALID_ARG;
+    if (d < 128 || d > 32768 || (d & 127)) return OGQ_ERR_UNSUPPORTED;
+    if (!(s == 2 || valid_orq_levels(s))) return OGQ_ERR_UNSUPPORTED;
+    if (total_elems > 0 && (!d_out || !aligned16(d_out))) return OGQ_ERR_INVALID_ARG;
+    if (total_elems == 0) return OGQ_OK;
+    const int sms = sm_count_of_current_device();
+    if (sms <= 0) return OGQ_ERR_CUDA;
+    cudaError_t e = ogq::launch_bucket_decode_sum(d_packed_k, d_levels_k, K, total_elems, d, s, scale, d_out, sms,
+                                                  (cudaStream_t)stream);
     return e == cudaSuccess ? OGQ_OK : OGQ_ERR_CUDA;
 }
 

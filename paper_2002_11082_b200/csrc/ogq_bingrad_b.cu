@@ -16,6 +16,8 @@
 
 namespace ogq {
 
+// CLIP: every value is first clamped to [-tau_arr[t], tau_arr[t]] (gradient clipping).
+template <bool CLIP>
 __global__ void __launch_bounds__(kThreads)
 k_bb_pass(const float* __restrict__ grad, const int64_t* __restrict__ off, int T, int64_t total,
           int64_t chunk, int pass, int lloyd_iters, const float* __restrict__ tau_arr, float* __restrict__ levels,
@@ -44,11 +46,11 @@ k_bb_pass(const float* __restrict__ grad, const int64_t* __restrict__ off, int T
     for_each_piece(off, T, lo, hi, [&](int t, int64_t tb, int64_t te, int64_t pb, int64_t pe) {
         if (pass > 0 && __ldcg(ws.done + t)) return;
         const float b0 = (pass == 0) ? -INFINITY : __ldcg(thresh + t);
-        const float tau = tau_arr ? __ldg(tau_arr + t) : INFINITY;  // clipping threshold (none: +Inf)
+        const float tau = CLIP ? __ldg(tau_arr + t) : 0.f;
         double s_lo = 0.0, s_hi = 0.0;
         long long c_lo = 0;
         visit_piece(grad, pb, pe, [&](float raw) {
-            const float v = copysignf(fminf(fabsf(raw), tau), raw);
+            const float v = CLIP ? copysignf(fminf(fabsf(raw), tau), raw) : raw;
             const bool below = v < b0;
             const double d = (double)v;
             s_lo += below ? d : 0.0;
@@ -141,8 +143,12 @@ cudaError_t launch_levels_bingrad_b(const float* d_grad, const int64_t* d_off, i
     if (e != cudaSuccess) return e;
     for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
         launch_begin("k_bb_pass", stream);
-        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, d_tau,
-                                                   d_levels, d_thresh, d_status, ws);
+        if (d_tau)
+            k_bb_pass<true><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, d_tau,
+                                                             d_levels, d_thresh, d_status, ws);
+        else
+            k_bb_pass<false><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, d_tau,
+                                                              d_levels, d_thresh, d_status, ws);
         launch_end(stream);
     }
     return cudaGetLastError();
@@ -195,8 +201,8 @@ cudaError_t launch_levels_bingrad_b_static(const float* d_grad, const int64_t* d
     if (e != cudaSuccess) return e;
     for (int pass = 0; pass <= lloyd_iters + 1; ++pass) {
         launch_begin("k_bb_pass", stream);
-        k_bb_pass<<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, nullptr,
-                                                   d_levels, d_thresh, d_status, ws);
+        k_bb_pass<false><<<g.ctas, kThreads, 0, stream>>>(d_grad, d_off, T, total, g.chunk, pass, lloyd_iters, nullptr,
+                                                          d_levels, d_thresh, d_status, ws);
         launch_end(stream);
     }
     return cudaGetLastError();

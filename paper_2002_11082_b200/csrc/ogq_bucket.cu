@@ -519,6 +519,106 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
     }
 }
 
+// Server step for fixed-length buckets: out[i] = scale * sum_k levels_k[i / d][code_k[i]].  Because d is
+// a multiple of 128, the packed codes of consecutive buckets form one contiguous bit stream (only the
+// last, shorter bucket is padded), so a warp takes 128 consecutive elements of the flat gradient at a
+// time and only has to fetch the level rows of the bucket they lie in.  Same additions in the same
+// (worker) order as ogq_unpack_sum with offsets j * d.
+constexpr int kDecWorkers = 8;  // workers per batch: their level rows and packed words are loaded before any is used
+
+template <int BITS>
+__global__ void __launch_bounds__(kThreads)
+k_bucket_decode_sum(const uint32_t* const* __restrict__ packed_k, const float* const* __restrict__ levels_k, int K,
+                    int64_t total, int d, int s, int64_t total_words, float scale, float* __restrict__ outp)
+{
+    __shared__ float sh_lv[kWarps][kDecWorkers][kMaxLevels];
+    __shared__ const uint32_t* sh_pk[kMaxWorkers];
+    __shared__ const float* sh_lp[kMaxWorkers];
+    for (int k = threadIdx.x; k < K; k += kThreads) { sh_pk[k] = packed_k[k]; sh_lp[k] = levels_k[k]; }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr uint32_t kMask4 = (BITS * 4 >= 32) ? 0xffffffffu : ((1u << (BITS * 4)) - 1u);
+    constexpr uint32_t kMask1 = (1u << BITS) - 1u;
+    const int64_t ngroups = (total + 127) >> 7;
+    for (int64_t g = (int64_t)blockIdx.x * kWarps + warp; g < ngroups; g += (int64_t)gridDim.x * kWarps) {
+        const int64_t i0 = (g << 7) + 4 * lane;
+        const int64_t j = (g << 7) / d;  // the bucket of this group
+        const int64_t bit = i0 * BITS;
+        const int64_t wi = bit >> 5;
+        const int sh = (int)(bit & 31);
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int k0 = 0; k0 < K; k0 += kDecWorkers) {
+            const int kn = (K - k0 < kDecWorkers) ? K - k0 : kDecWorkers;
+            // all loads of the batch first (level rows: every code a BITS-bit field can hold gets an entry)
+            float row[kDecWorkers];
+            uint32_t w_lo[kDecWorkers], w_hi[kDecWorkers];
+            const bool straddle = sh + 4 * BITS > 32;
+#pragma unroll
+            for (int u = 0; u < kDecWorkers; ++u) {
+                row[u] = 0.f; w_lo[u] = 0u; w_hi[u] = 0u;
+                if (u < kn) {
+                    row[u] = __ldg(sh_lp[k0 + u] + j * s + (lane < s ? lane : s - 1));
+                    if (i0 < total) {
+                        const uint32_t* p = sh_pk[k0 + u];
+                        if (wi < total_words) w_lo[u] = __ldg(p + wi);
+                        if (straddle && wi + 1 < total_words) w_hi[u] = __ldg(p + wi + 1);
+                    }
+                }
+            }
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < kDecWorkers; ++u)
+                if (u < kn) sh_lv[warp][u][lane] = row[u];
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < kDecWorkers; ++u) {
+                if (u < kn) {
+                    const uint32_t bits4 = __funnelshift_r(w_lo[u], w_hi[u], sh) & kMask4;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        acc[e] = __fadd_rn(acc[e], sh_lv[warp][u][(bits4 >> (e * BITS)) & kMask1]);
+                }
+            }
+        }
+        if (i0 + 3 < total) {
+            *reinterpret_cast<float4*>(outp + i0) = make_float4(__fmul_rn(acc[0], scale), __fmul_rn(acc[1], scale),
+                                                                __fmul_rn(acc[2], scale), __fmul_rn(acc[3], scale));
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (i0 + e < total) outp[i0 + e] = __fmul_rn(acc[e], scale);
+        }
+    }
+}
+
+cudaError_t launch_bucket_decode_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                                     int64_t total, int d, int s, float scale, float* d_out, int sm_count,
+                                     cudaStream_t stream)
+{
+    const int bits = ogq_bits_for_levels(s);
+    const int64_t nb = (total + d - 1) / d;
+    const int64_t last = total - (nb - 1) * d;
+    const int64_t total_words = (nb - 1) * ((int64_t)d * bits / 32) + ((last * bits + 31) / 32 + 3) / 4 * 4;
+    const int64_t ngroups = (total + 127) >> 7;
+    int64_t ctas = (ngroups + kWarps - 1) / kWarps;
+    if (ctas > (int64_t)sm_count * 8) ctas = (int64_t)sm_count * 8;
+    launch_begin("k_bucket_decode_sum", stream);
+#define OGQ_LAUNCH_BD(B)                                                                                        \
+    k_bucket_decode_sum<B><<<(int)ctas, kThreads, 0, stream>>>(d_packed_k, d_levels_k, K, total, d, s, total_words, \
+                                                               scale, d_out)
+    switch (bits) {
+        case 1: OGQ_LAUNCH_BD(1); break;
+        case 2: OGQ_LAUNCH_BD(2); break;
+        case 3: OGQ_LAUNCH_BD(3); break;
+        case 4: OGQ_LAUNCH_BD(4); break;
+        case 5: OGQ_LAUNCH_BD(5); break;
+        default: return cudaErrorInvalidValue;
+    }
+#undef OGQ_LAUNCH_BD
+    launch_end(stream);
+    return cudaGetLastError();
+}
+
 static int bkt_pow2(int d);
 
 static size_t bkt_smem_bytes(int d)

@@ -50,6 +50,9 @@ cudaError_t launch_bucket_encode(const float* d_grad, int64_t total, int d, int 
 cudaError_t launch_quant_error(const float* d_grad, const int64_t* d_off, int T, int64_t total, int s,
                                const float* d_levels, const int64_t* d_packed_off, const uint32_t* d_packed,
                                double* d_err, int sm_count, cudaStream_t stream);
+cudaError_t launch_bucket_decode_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
+                                     int64_t total, int d, int s, float scale, float* d_out, int sm_count,
+                                     cudaStream_t stream);
 int dense_digits(int s);  // codes per 32-bit word of the base-s format (0: unsupported s)
 cudaError_t launch_quantize_pack_dense(const float* d_grad, const int64_t* d_off, int T, int64_t total, int s,
                                        const float* d_levels, uint64_t seed, uint32_t stream_id,

@@ -8,8 +8,13 @@
 // prefix sums into a few narrow candidate intervals.  Round 2 streams the bucket
 // again, copies the few percent of elements inside the intervals to scratch and
 // histograms them on a finer grid; round 3 and later work on the copied keys
-// only, until every level's rank falls into a single-key cell.  Tensors of at
-// most kSmallN elements are sorted in shared memory instead.
+// only, until every level's rank falls into a single-key cell.  As soon as the
+// elements still in question fit one shared-memory sort, the next pass only
+// copies them and the tensor is finished from the sorted keys.  Tensors of at
+// most kSmallN elements are sorted in shared memory right away; mid-size ones
+// run on a CTA of their own (round 1 in the first launch, the rest in the
+// second).  The key buffers hold one eighth of the bucket: a pass whose copies
+// do not fit is repeated on the gradient with the narrower intervals.
 //
 // All cross-CTA accumulation is integer (atomic adds, min, max), and the
 // per-tensor prefix sums are built in a fixed order, so results are
@@ -2271,12 +2276,13 @@ cudaError_t launch_levels_select(const float* d_grad, const int64_t* d_off, int 
     // Flat streaming CTAs: one wave (kSelResident per SM).  Each CTA pays a set-up, a flush of its
     // cells and an arrival per tensor piece, so larger chunks stream more of the time; a second wave
     // balanced a lone call slightly better in round 1 but cost throughput whenever several calls
-    // (workers on their own streams) share the GPU.  Chunks are at least 131,072 elements: on a bucket of
-    // 25 M elements that leaves a third of the wave's slots to concurrent calls (measured with eight
-    // workers in flight: 8 % more throughput, 3 % slower alone).
+    // (workers on their own streams) share the GPU.  Buckets above 4 M elements get chunks of at least
+    // 131,072 elements: on a bucket of 25 M elements that leaves a third of the wave's slots to concurrent
+    // calls (measured with eight workers in flight: 8 % more throughput, 3 % slower alone); smaller
+    // buckets keep 32,768, where a lone call is all that matters.
     const int64_t wave = (int64_t)kSelResident * sm_count;
     const int target = wave < kMaxFlatCtas ? (int)wave : kMaxFlatCtas;
-    FlatGrid g = make_flat_grid(total, target, 131072);
+    FlatGrid g = make_flat_grid(total, target, total > ((int64_t)1 << 22) ? 131072 : 32768);
     SelArgs A;
     A.grad = d_grad; A.tau = d_tau; A.off = d_off; A.T = T; A.total = total; A.chunk = g.chunk; A.flat_ctas = g.ctas;
     A.scheme = scheme; A.s = s; A.levels = d_levels; A.status = d_status;

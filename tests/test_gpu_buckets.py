@@ -152,3 +152,35 @@ def test_bucket_mode_special_buckets_and_argument_checks():
         ogq.ogq_bucket_encode(z, 1024, 128, ogq.OGQ_ORQ, 4, 0, 0.0, 0, 0, z, z, i, i)
     ogq.ogq_bucket_encode(z, 0, 128, ogq.OGQ_ORQ, 9, 0, 0.0, 0, 0, z, z, i, i)  # nothing to do
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("s,d", [(9, 512), (3, 2048), (5, 256), (17, 128), (2, 1024)])
+def test_bucket_decode_sum_equals_unpack_sum_with_offsets_jd(s, d):
+    """K workers encoded in bucket mode, summed by ogq_bucket_decode_sum: equal to the oracle's sum over
+    the same packed buffers and to ogq_unpack_sum called with offsets j * d (bit for bit: same additions)."""
+    dev = torch.device("cuda:0")
+    K = 5
+    total = 300_000 + 77
+    off = bucket_offsets(total, d)
+    scheme = ogq.OGQ_BINGRAD_B if s == 2 else ogq.OGQ_ORQ
+    lvs, pks = [], []
+    for k in range(K):
+        v = wl.laplace(np.random.Generator(np.random.PCG64(90 + k)), total, 1e-3 * (1 + k))
+        lv, th, st, packed = run_encode(v, d, scheme, s, 0, seed=2, stream_id=k)
+        lvs.append(lv)
+        pks.append(packed)
+    d_lv = [torch.from_numpy(l).to(dev) for l in lvs]
+    d_pk = [torch.from_numpy(p.view(np.int32)).to(dev) for p in pks]
+    pad = 64
+    buf = torch.full((total + 2 * pad,), 12345.0, device=dev)
+    ogq.ogq_bucket_decode_sum(ogq.device_pointer_array(d_pk), ogq.device_pointer_array(d_lv), K, total, d, s, 1.0 / K,
+                              buf[pad : pad + total])
+    torch.cuda.synchronize()
+    h = buf.cpu().numpy()
+    assert np.all(h[:pad] == 12345.0) and np.all(h[pad + total :] == 12345.0), "canary overwritten"
+    got = h[pad : pad + total]
+    want = oracle.bucket_unpack_sum(pks, lvs, off, s, 1.0 / K)
+    tol = 1e-5 * float(np.max(np.abs(want)))
+    assert np.all(np.abs(got.astype(np.float64) - want) <= tol)
+    db = DeviceBucket(np.zeros(total, np.float32), off)
+    assert np.array_equal(got, db.unpack_sum(pks, lvs, s, 1.0 / K))

@@ -355,3 +355,24 @@ def test_resnet50_eight_workers_on_eight_streams():
         assert np.array_equal(serial[1][k], together[1][k]), k
     want, _ = oracle.bucket_levels_orq(b.values, b.offsets, s)
     assert levels_close(together[0][0], want)
+
+
+def test_orq_levels_when_the_rank_target_is_an_exact_integer():
+    """A uniform grid of 17 values, each repeated 2^16 times (1.1 M elements): every T of Algorithm 1 is an
+    integer up to fp64 rounding, so two neighbouring data values satisfy the discrete condition equally.
+    The levels must be grid values that satisfy it (either choice), and the codes must match the oracle's
+    for the levels returned."""
+    reps = 1 << 16
+    grid = (np.arange(17, dtype=np.float32) - 8.0) / np.float32(1024.0)
+    v = np.repeat(grid, reps)
+    np.random.Generator(np.random.PCG64(5)).shuffle(v)
+    off = np.array([0, v.size], np.int64)
+    db = DeviceBucket(v, off)
+    view = SortedView(v)
+    for s in (3, 5, 9, 17):
+        lv, st = db.levels_orq(s)
+        assert st[0] == 0 and np.all(np.isin(lv[0], grid))
+        check_orq_levels_by_condition(v, lv[0], view)
+        got, _ = db.quantize_pack(ogq.OGQ_ORQ, s, lv, None, 3, 0)
+        want, _ = oracle.bucket_quantize_pack(v, off, oracle.ORQ, s, lv, None, 3, 0)
+        assert np.array_equal(got, want)
