@@ -40,7 +40,7 @@ constexpr int kSelM = 7;           // log2(cells per binade) in the window
 constexpr int kSmallN = 4096;      // tensors up to this size are sorted in shared memory
 constexpr int kMidN = 131072;      // tensors up to this size are solved start to finish by one CTA of their own
 constexpr int kStageCap = 320;     // per-warp staging entries for compaction
-constexpr int kParkMax = 256;      // values one warp can park between two checks of round 2 (32 lanes x 8)
+constexpr int kParkMax = 256;      // values one warp can park between two checks in the tail of round 2 (32 lanes x 8)
 constexpr int kMaxSlices = 64;     // CTAs that share one tensor's copied keys in round 3
 constexpr int kSliceElems = 16384;
 constexpr int kMaxRounds = 32;
@@ -370,7 +370,7 @@ __device__ __forceinline__ uint32_t atom_shared_add(uint32_t addr, uint32_t v)
 
 constexpr int kPackedPerSign = kSelW << kSelM;  // fine cells per sign (2048)
 constexpr int kPackedCells = 2 * kPackedPerSign;
-constexpr int kPackTrips = 4;                    // loop trips between two folds of the packed cells
+constexpr int kPackTrips = 8;                    // loop trips between two folds of the packed cells
 static_assert(kPackedCells * sizeof(uint32_t) <= kSelWarps * kStageCap * sizeof(uint32_t),
               "the packed cells live in the (otherwise unused) compaction stages during round 1");
 
@@ -419,7 +419,11 @@ struct Round1Body {
     // together with multiply-adds and the sign is not branched on.
     __device__ __forceinline__ void fine_packed(uint32_t bits, uint32_t r2)
     {
-        uint32_t addr = pk + ((r2 >> (24 - kSelM - 2)) & ((uint32_t)(kPackedPerSign - 1) << 2));
+        // pk + 4 * cell, cell = r2 >> (24 - kSelM): the high half of a multiply-add by a power of two,
+        // which the compiler turns into one shift-and-add
+        static_assert(kSelM == 7, "the shift below is 32 - (24 - kSelM - 2)");
+        uint32_t addr;
+        asm("mad.hi.u32 %0, %1, 131072, %2;" : "=r"(addr) : "r"(r2 & ~((1u << (24 - kSelM)) - 1u)), "r"(pk));
         if (!MAG) asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(addr) : "r"(bits >> 31), "r"(4u * kPackedPerSign));
         red_shared_add(addr, (bits & ((1u << (23 - kSelM)) - 1u)) | one24);
     }
@@ -675,10 +679,14 @@ struct Round2Warp {
         const uint32_t pos = atom_shared_add(fillp, 1u);
         asm volatile("st.shared.u32 [%0], %1;" :: "r"(stage + (pos << 2)), "r"(bits) : "memory");
     }
+    // Word address = coarse + ((bits & ~(2^22 - 1)) >> 20), written as the high half of a multiply-add
+    // by 2^12: the compiler makes one shift-and-add of it (a real multiplication, with the factor
+    // hidden in a kernel argument, was measured slower).  The funnel shift takes its count modulo 32.
     __device__ __forceinline__ uint32_t top_is_hit(uint32_t bits) const
     {
-        uint32_t word;
-        asm("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(coarse + ((bits >> 20) & 0xffcu)));
+        uint32_t addr, word;
+        asm("mad.hi.u32 %0, %1, 4096, %2;" : "=r"(addr) : "r"(bits & 0xffc00000u), "r"(coarse));
+        asm("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(addr));
         return __funnelshift_l(0u, word, bits >> 17);  // the block's bit is now bit 31
     }
     __device__ __forceinline__ void one(float v)
@@ -691,16 +699,16 @@ struct Round2Warp {
     {
         hits = __funnelshift_l(top_is_hit(__float_as_uint(clip(v))), hits, 1);
     }
-    // Parks the elements marked in `hits` (bit 7 = the first of the eight elements tested: p[0].x,
-    // ..., p[0].w, p[stride].x, ...).  The values are read again, from L1: a hit is rare, and a
-    // register cannot be picked by a run-time index.
+    // Parks the elements marked in `hits` (bit 15 = the first of the sixteen elements tested: p[0].x,
+    // ..., p[0].w, p[stride].x, ..., p[3 * stride].w).  The values are read again, from L1: a hit is
+    // rare, and a register cannot be picked by a run-time index.
     __device__ __forceinline__ void park_hits(uint32_t hits, const float4* p, int stride)
     {
         while (hits) {
             const int b = 31 - __clz(hits);
             hits &= ~(1u << b);
-            const int j = 7 - b;
-            const float* src = reinterpret_cast<const float*>(p + ((j & 4) ? stride : 0)) + (j & 3);
+            const int j = 15 - b;
+            const float* src = reinterpret_cast<const float*>(p + (j >> 2) * stride) + (j & 3);
             park(__float_as_uint(clip(__ldg(src))));
         }
     }
@@ -739,7 +747,7 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
         else if (lane >= 4 && lane - 4 < (int)(pe - b)) w.one(__ldg(grad + b + lane - 4));
         __syncwarp();
     }
-    // at most kParkMax values are parked between two checks
+    // The tail below parks at most kParkMax values between two checks of the stage's fill.
     auto check = [&]() {
         __syncwarp();
         const int f = *(volatile int*)&fills[warp];
@@ -754,23 +762,48 @@ __device__ __noinline__ void stream_round2(const float* __restrict__ grad, int64
     int64_t i0 = (a >> 2) + warp * 32;  // the trip counts below are warp-uniform
     // Trips of 4 x kSelThreads float4 (one contiguous block of kTripBytes per CTA).  One thread asks
     // L2 for the block kPrefetchTrips ahead, so that the loads below find their lines there.
+    // A lane tests its sixteen values of a trip without branching; the warp then parks the trip's
+    // hits in one go (nearly every trip has a hit in some lane, so the divergent parking code is
+    // paid once per trip, not once per few values).  `fill` mirrors the stage's fill counter in a
+    // register: it is the same in all lanes, so whether to drain first is a uniform decision.
     int64_t pf = (a >> 2) + (int64_t)kPrefetchTrips * 4 * kSelThreads;
+    __syncwarp();
+    int fill = *(volatile int*)&fills[warp];
     for (; i0 + 3 * kSelThreads + 32 <= e; i0 += 4 * kSelThreads) {
         if (threadIdx.x == 0 && pf + 4 * kSelThreads <= e) prefetch_l2(g4 + pf, kTripBytes);
         pf += 4 * kSelThreads;
         float4 x[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i0 + lane + u * kSelThreads);
+        uint32_t hits = 0u;
 #pragma unroll
-        for (int h = 0; h < 4; h += 2) {
-            uint32_t hits = 0u;
-            w.test(x[h].x, hits); w.test(x[h].y, hits); w.test(x[h].z, hits); w.test(x[h].w, hits);
-            w.test(x[h + 1].x, hits); w.test(x[h + 1].y, hits); w.test(x[h + 1].z, hits); w.test(x[h + 1].w, hits);
-            if (hits) w.park_hits(hits, g4 + i0 + lane + h * kSelThreads, kSelThreads);
-            check();
+        for (int u = 0; u < 4; ++u) {
+            w.test(x[u].x, hits); w.test(x[u].y, hits); w.test(x[u].z, hits); w.test(x[u].w, hits);
+        }
+        for (;;) {  // one turn, unless the stage has to be drained to make room
+            const int tot = (int)__reduce_add_sync(0xffffffffu, (uint32_t)__popc(hits));
+            if (tot == 0) break;
+            if (fill + tot <= kStageCap) {
+                if (hits) w.park_hits(hits, g4 + i0 + lane, kSelThreads);
+                fill += tot;
+                break;
+            }
+            if (fill) {
+                round2_drain(&tb, &ctx, stage, fill);
+                if (lane == 0) fills[warp] = 0;
+                __syncwarp();
+                fill = 0;
+                continue;
+            }
+            // more hits in one trip than the empty stage holds: the first eight values of every lane now
+            const uint32_t first = hits & 0xff00u;
+            if (first) w.park_hits(first, g4 + i0 + lane, kSelThreads);
+            fill = (int)__reduce_add_sync(0xffffffffu, (uint32_t)__popc(first));
+            hits &= 0xffu;
         }
     }
     if (i0 < e) {
+        check();  // the trips above may have left the stage nearly full
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int64_t i = i0 + lane + (int64_t)u * kSelThreads;
@@ -1878,7 +1911,6 @@ __device__ void finish_alone(const SelArgs& A, int t, unsigned char* smem, Table
 __global__ void __launch_bounds__(kSelThreads, kSelResident) k_sel_round1(SelArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    __shared__ Table tb;
     __shared__ SolverShared S;
     __shared__ Interval r1iv[kMaxIv];
     __shared__ int sh_i[kSelWarps];
