@@ -521,33 +521,43 @@ __device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64
     const float4* g4 = reinterpret_cast<const float4*>(grad);
     const int64_t first = a >> 2, e = b >> 2;
     const int64_t ntrips = (e - first) / (4 * kSelThreads);  // full trips: the same for every thread
-    int64_t pf = first + (int64_t)kPrefetchTrips * 4 * kSelThreads;
     constexpr int kNp = MAG ? kPackedPerSign : kPackedCells;
+    const float4* src = g4 + first + tid;                                              // this thread's next load
+    const float4* pfp = g4 + first + (int64_t)kPrefetchTrips * 4 * kSelThreads;       // next block to ask L2 for
+    const float4* const pf_end = g4 + e - 4 * kSelThreads;
     for (int64_t t0 = 0; t0 < ntrips; t0 += kPackTrips) {
         const int nt = (int)((ntrips - t0 < kPackTrips) ? ntrips - t0 : kPackTrips);
         if (tid == 0) { sh_coarse = 0u; sh_total = 0u; }
         __syncthreads();
+        const float4* const period = src;
         for (int tt = 0; tt < nt; ++tt) {
-            const int64_t i = first + (t0 + tt) * 4 * kSelThreads + tid;
-            if (tid == 0 && pf + 4 * kSelThreads <= e) prefetch_l2(g4 + pf, kTripBytes);
-            pf += 4 * kSelThreads;
+            if (tid == 0 && pfp <= pf_end) prefetch_l2(pfp, kTripBytes);
+            pfp += 4 * kSelThreads;
             float4 x[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) x[u] = __ldg(g4 + i + u * kSelThreads);
+            for (int u = 0; u < 4; ++u) x[u] = __ldg(src + u * kSelThreads);
+            src += 4 * kSelThreads;
 #pragma unroll
             for (int u = 0; u < 4; ++u) f.template four<true>(x[u]);
         }
         __syncthreads();
         // fold, phase 1: do the packed counts add up to the values that went in?
         uint32_t mine = 0u;
-        for (int p = tid; p < kNp; p += kSelThreads) mine += packed[p] >> 24;
+        uint32_t wv[kNp / kSelThreads];  // this thread's packed words, read once
+#pragma unroll
+        for (int k = 0; k < kNp / kSelThreads; ++k) {
+            wv[k] = packed[tid + k * kSelThreads];
+            mine += wv[k] >> 24;
+        }
         mine = __reduce_add_sync(0xffffffffu, mine);
         if ((tid & 31) == 0 && mine) atomicAdd(&sh_total, mine);
         __syncthreads();
         const bool ok = sh_total + sh_coarse == (uint32_t)nt * 16u * kSelThreads;
         // phase 2: into the wide counters (packed index p: negative values mirror below the middle)
-        for (int p = tid; p < kNp; p += kSelThreads) {
-            const uint32_t w = packed[p];
+#pragma unroll
+        for (int k = 0; k < kNp / kSelThreads; ++k) {
+            const int p = tid + k * kSelThreads;
+            const uint32_t w = wv[k];
             if (w) {
                 packed[p] = 0u;
                 if (ok) {
@@ -569,10 +579,9 @@ __device__ __noinline__ void stream_round1(const float* __restrict__ grad, int64
             // the window were counted directly the first time and are skipped now)
             __syncthreads();
             for (int tt = 0; tt < nt; ++tt) {
-                const int64_t i = first + (t0 + tt) * 4 * kSelThreads + tid;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const float4 x = __ldg(g4 + i + u * kSelThreads);
+                    const float4 x = __ldg(period + (tt * 4 + u) * kSelThreads);
                     const float vv[4] = {f.canon(x.x), f.canon(x.y), f.canon(x.z), f.canon(x.w)};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
