@@ -63,7 +63,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             if verbose:
                 print(res.stderr, end="")
     objs = [_obj(s) for s in sources()]
-    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB_PATH] + objs, check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB_PATH] + objs + ["-ldl"], check=True)
     return LIB_PATH
 
 

@@ -1,5 +1,6 @@
 // extern "C" entry points: argument validation, scratch layout, kernel launches.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <string.h>
 
 #include <atomic>
@@ -50,6 +51,15 @@ int sm_count_of_current_device()
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// One NVTX range per data-path call, named after the entry point (a stage of the path on a profiler's
+// host timeline; a no-op when no tool is attached).
+struct StageRange {
+    explicit StageRange(const char* name) { nvtxRangePushA(name); }
+    ~StageRange() { nvtxRangePop(); }
+    StageRange(const StageRange&) = delete;
+    StageRange& operator=(const StageRange&) = delete;
+};
 
 bool valid_orq_levels(int s) { return s == 3 || s == 5 || s == 9 || s == 17; }
 
@@ -157,6 +167,7 @@ ogq_status ogq_levels_bingrad(const float* d_grad, const int64_t* d_off, int T, 
                               int variant, int lloyd_iters, float* d_levels, float* d_thresh,
                               int32_t* d_status, void* d_ws, size_t ws_bytes, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_levels_bingrad");
     return levels_bingrad_impl(d_grad, d_off, T, total_elems, variant, lloyd_iters, nullptr, d_levels, d_thresh,
                                d_status, d_ws, ws_bytes, stream);
 }
@@ -166,6 +177,7 @@ ogq_status ogq_levels_bingrad_clipped(const float* d_grad, const int64_t* d_off,
                                       float* d_thresh, int32_t* d_status, void* d_ws, size_t ws_bytes,
                                       ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_levels_bingrad_clipped");
     if (!d_tau) return OGQ_ERR_INVALID_ARG;
     return levels_bingrad_impl(d_grad, d_off, T, total_elems, variant, lloyd_iters, d_tau, d_levels, d_thresh,
                                d_status, d_ws, ws_bytes, stream);
@@ -174,6 +186,7 @@ ogq_status ogq_levels_bingrad_clipped(const float* d_grad, const int64_t* d_off,
 ogq_status ogq_clip_threshold(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, float c,
                               float* d_tau, int32_t* d_status, void* d_ws, size_t ws_bytes, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_clip_threshold");
     if (T < 0 || total_elems < 0 || !d_off || !d_tau || !d_status || !(c > 0.f) || !(c < 1e30f))
         return OGQ_ERR_INVALID_ARG;
     if (total_elems > 0 && (!d_grad || !aligned16(d_grad))) return OGQ_ERR_INVALID_ARG;
@@ -190,6 +203,7 @@ ogq_status ogq_levels_bingrad_b_noalloc(const float* d_grad, const int64_t* d_of
                                         int lloyd_iters, float* d_levels, float* d_thresh,
                                         int32_t* d_status, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_levels_bingrad_b_noalloc");
     if (T < 0 || total_elems < 0 || !d_off || !d_levels || !d_thresh || !d_status || lloyd_iters < 0 ||
         lloyd_iters > 1024)
         return OGQ_ERR_INVALID_ARG;
@@ -224,6 +238,7 @@ ogq_status ogq_levels_orq(const float* d_grad, const int64_t* d_off, int T, int6
                           float* d_levels, int32_t* d_status, void* d_ws, size_t ws_bytes,
                           ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_levels_orq");
     return levels_orq_impl(d_grad, d_off, T, total_elems, s, nullptr, d_levels, d_status, d_ws, ws_bytes, stream);
 }
 
@@ -231,6 +246,7 @@ ogq_status ogq_levels_orq_clipped(const float* d_grad, const int64_t* d_off, int
                                   const float* d_tau, float* d_levels, int32_t* d_status, void* d_ws,
                                   size_t ws_bytes, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_levels_orq_clipped");
     if (!d_tau) return OGQ_ERR_INVALID_ARG;
     return levels_orq_impl(d_grad, d_off, T, total_elems, s, d_tau, d_levels, d_status, d_ws, ws_bytes, stream);
 }
@@ -269,6 +285,7 @@ ogq_status ogq_quantize_pack(const float* d_grad, const int64_t* d_off, int T, i
                              uint64_t seed, uint32_t stream_id, const int64_t* d_packed_off,
                              uint32_t* d_packed, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_quantize_pack");
     return quantize_pack_impl(d_grad, d_off, T, total_elems, scheme, s, d_levels, d_thresh, nullptr, seed,
                               stream_id, d_packed_off, d_packed, stream);
 }
@@ -278,6 +295,7 @@ ogq_status ogq_quantize_pack_clipped(const float* d_grad, const int64_t* d_off, 
                                      const float* d_tau, uint64_t seed, uint32_t stream_id,
                                      const int64_t* d_packed_off, uint32_t* d_packed, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_quantize_pack_clipped");
     if (!d_tau) return OGQ_ERR_INVALID_ARG;
     return quantize_pack_impl(d_grad, d_off, T, total_elems, scheme, s, d_levels, d_thresh, d_tau, seed,
                               stream_id, d_packed_off, d_packed, stream);
@@ -287,6 +305,7 @@ ogq_status ogq_unpack_sum(const uint32_t* const* d_packed_k, const float* const*
                           const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total_elems,
                           int s, float scale, float* d_out, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_unpack_sum");
     if (T < 0 || total_elems < 0 || !d_off || !d_packed_off || !d_packed_k || !d_levels_k)
         return OGQ_ERR_INVALID_ARG;
     if (K < 1 || K > 64) return OGQ_ERR_INVALID_ARG;
@@ -320,12 +339,14 @@ ogq_status ogq_quant_error(const float* d_grad, const int64_t* d_off, int T, int
                            const float* d_levels, const int64_t* d_packed_off, const uint32_t* d_packed,
                            double* d_err, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_quant_error");
     return quant_error_impl(d_grad, d_off, T, total_elems, s, d_levels, d_packed_off, d_packed, true, d_err, stream);
 }
 
 ogq_status ogq_expected_error(const float* d_grad, const int64_t* d_off, int T, int64_t total_elems, int s,
                               const float* d_levels, double* d_err, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_expected_error");
     return quant_error_impl(d_grad, d_off, T, total_elems, s, d_levels, nullptr, nullptr, false, d_err, stream);
 }
 
@@ -350,6 +371,7 @@ ogq_status ogq_quantize_pack_dense(const float* d_grad, const int64_t* d_off, in
                                    const float* d_levels, uint64_t seed, uint32_t stream_id,
                                    const int64_t* d_packed_off, uint32_t* d_packed, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_quantize_pack_dense");
     if (T < 0 || total_elems < 0 || !d_off || !d_packed_off || !d_levels) return OGQ_ERR_INVALID_ARG;
     if (!valid_orq_levels(s)) return OGQ_ERR_UNSUPPORTED;
     if (total_elems > 0 && (!d_grad || !d_packed || !aligned16(d_grad) || !aligned16(d_packed)))
@@ -366,6 +388,7 @@ ogq_status ogq_unpack_sum_dense(const uint32_t* const* d_packed_k, const float* 
                                 const int64_t* d_off, const int64_t* d_packed_off, int T, int64_t total_elems,
                                 int s, float scale, float* d_out, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_unpack_sum_dense");
     if (T < 0 || total_elems < 0 || !d_off || !d_packed_off || !d_packed_k || !d_levels_k)
         return OGQ_ERR_INVALID_ARG;
     if (K < 1 || K > 64) return OGQ_ERR_INVALID_ARG;
@@ -393,6 +416,7 @@ ogq_status ogq_bucket_encode(const float* d_grad, int64_t total_elems, int d, og
                              float clip_c, uint64_t seed, uint32_t stream_id, float* d_levels, float* d_thresh,
                              int32_t* d_status, uint32_t* d_packed, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_bucket_encode");
     if (total_elems < 0 || iters < 0 || iters > 1024 || !d_levels || !d_status || !(clip_c >= 0.f) || !(clip_c < 1e30f))
         return OGQ_ERR_INVALID_ARG;
     if (d < 128 || d > 32768 || (d & 127)) return OGQ_ERR_UNSUPPORTED;
@@ -420,6 +444,7 @@ ogq_status ogq_bucket_encode(const float* d_grad, int64_t total_elems, int d, og
 ogq_status ogq_bucket_decode_sum(const uint32_t* const* d_packed_k, const float* const* d_levels_k, int K,
                                  int64_t total_elems, int d, int s, float scale, float* d_out, ogq_stream_t stream)
 {
+    StageRange nvtx_range("ogq_bucket_decode_sum");
     if (total_elems < 0 || !d_packed_k || !d_levels_k) return OGQ_ERR_INVALID_ARG;
     if (K < 1 || K > 64) return OGQ_ERR_INVALID_ARG;
     if (d < 128 || d > 32768 || (d & 127)) return OGQ_ERR_UNSUPPORTED;
