@@ -51,33 +51,6 @@ __device__ __forceinline__ void bkt_cmpx(uint32_t& a, uint32_t& b)
     b = hi;
 }
 
-template <int KPT, int K2>
-__device__ __forceinline__ void bkt_flip_local(uint32_t (&r)[KPT], int k)
-{
-    if constexpr (K2 >= 2) {
-        if (k == K2) {
-#pragma unroll
-            for (int e = 0; e < KPT; ++e)
-                if ((e & (K2 / 2)) == 0) bkt_cmpx(r[e], r[e ^ (K2 - 1)]);
-        } else {
-            bkt_flip_local<KPT, K2 / 2>(r, k);
-        }
-    }
-}
-
-template <int KPT, int J>
-__device__ __forceinline__ void bkt_halve_local(uint32_t (&r)[KPT], int k)
-{
-    if constexpr (J >= 1) {
-        if (4 * J <= k) {
-#pragma unroll
-            for (int e = 0; e < KPT; ++e)
-                if ((e & J) == 0) bkt_cmpx(r[e], r[e | J]);
-        }
-        bkt_halve_local<KPT, J / 2>(r, k);
-    }
-}
-
 // Exchange with thread t ^ m: this thread's register e against the partner's register e (REV false)
 // or KPT - 1 - e (REV true); the thread on the lower side keeps the smaller keys.
 template <int KPT, bool REV>
@@ -96,23 +69,71 @@ __device__ __forceinline__ void bkt_cross(uint32_t (&r)[KPT], uint32_t* xch, int
 #pragma unroll
         for (int e = 0; e < KPT; ++e) o[e] = xch[(REV ? KPT - 1 - e : e) * nt + (t ^ m)];
     }
+    // the side of the exchange decides once whether this thread keeps minima or maxima: one predicated
+    // instruction pair per key instead of a minimum, a maximum and a select
 #pragma unroll
-    for (int e = 0; e < KPT; ++e) r[e] = keep_min ? min(r[e], o[e]) : max(r[e], o[e]);
+    for (int e = 0; e < KPT; ++e)
+        asm("{ .reg .pred p; setp.ne.u32 p, %2, 0; @p min.u32 %0, %0, %1; @!p max.u32 %0, %0, %1; }"
+            : "+r"(r[e]) : "r"(o[e]), "r"((uint32_t)keep_min));
+}
+
+// The stages of a merge that stay inside a warp, written out at compile time (no run-time dispatch on
+// the merge size, so the registers never have to be moved between code paths): halvings at lane
+// distances 16 ... 1 (FROM_LANES) or only those inside a thread's registers.
+template <int KPT, bool FROM_LANES>
+__device__ __forceinline__ void bkt_merge_tail(uint32_t (&r)[KPT], uint32_t* xch)
+{
+    const int t = threadIdx.x;
+    if constexpr (FROM_LANES) {
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) bkt_cross<KPT, false>(r, xch, m, (t & m) == 0);
+    }
+#pragma unroll
+    for (int j = KPT / 2; j >= 1; j >>= 1) {
+#pragma unroll
+        for (int e = 0; e < KPT; ++e)
+            if ((e & j) == 0) bkt_cmpx(r[e], r[e | j]);
+    }
+}
+
+// Sorts the 32 * KPT keys of every warp ascending: the whole network unrolled at compile time.
+template <int KPT>
+__device__ __forceinline__ void bkt_sort_warp(uint32_t (&r)[KPT], uint32_t* xch)
+{
+    const int t = threadIdx.x;
+#pragma unroll
+    for (int k = 2; k <= 32 * KPT; k <<= 1) {
+        if (k <= KPT) {
+#pragma unroll
+            for (int e = 0; e < KPT; ++e)
+                if ((e & (k >> 1)) == 0) bkt_cmpx(r[e], r[e ^ (k - 1)]);
+#pragma unroll
+            for (int j = k >> 2; j >= 1; j >>= 1) {
+#pragma unroll
+                for (int e = 0; e < KPT; ++e)
+                    if ((e & j) == 0) bkt_cmpx(r[e], r[e | j]);
+            }
+        } else {
+            const int m = k / KPT - 1;  // flip: lane t against t ^ m, registers reversed
+            bkt_cross<KPT, true>(r, xch, m, (t & ((m + 1) >> 1)) == 0);
+#pragma unroll
+            for (int j = k >> 2; j >= KPT; j >>= 1) bkt_cross<KPT, false>(r, xch, j / KPT, (t & (j / KPT)) == 0);
+            bkt_merge_tail<KPT, false>(r, xch);
+        }
+    }
 }
 
 template <int KPT>
 __device__ __forceinline__ void bkt_sort_regs(uint32_t (&r)[KPT], uint32_t* xch, int P)
 {
     const int t = threadIdx.x;
-    for (int k = 2; k <= P; k <<= 1) {
-        if (k <= KPT) {
-            bkt_flip_local<KPT, KPT>(r, k);
-        } else {
-            const int m = k / KPT - 1;  // flip: thread t against t ^ m, registers reversed
-            bkt_cross<KPT, true>(r, xch, m, (t & ((m + 1) >> 1)) == 0);
-            for (int j = k >> 2; j >= KPT; j >>= 1) bkt_cross<KPT, false>(r, xch, j / KPT, (t & (j / KPT)) == 0);
-        }
-        bkt_halve_local<KPT, KPT / 2>(r, k);
+    bkt_sort_warp<KPT>(r, xch);
+    // merges across warps: the flip and the halvings at 32 threads or more go through shared memory
+    for (int k = 64 * KPT; k <= P; k <<= 1) {
+        const int m = k / KPT - 1;
+        bkt_cross<KPT, true>(r, xch, m, (t & ((m + 1) >> 1)) == 0);
+        for (int j = k >> 2; j >= 32 * KPT; j >>= 1) bkt_cross<KPT, false>(r, xch, j / KPT, (t & (j / KPT)) == 0);
+        bkt_merge_tail<KPT, true>(r, xch);
     }
 }
 
@@ -163,6 +184,52 @@ __device__ __forceinline__ uint32_t bkt_qstar_prefix(const uint32_t* keys, const
     if (k < 0) k = 0;
     if (k > m - 1) k = m - 1;
     return keys[i1 - 1 - (int)k];
+}
+
+// One depth of Algorithm 1 for a bucket held by ONE warp, called by all its lanes with the sorted keys
+// still in their registers.  The positions of the brackets come from counting (a compare per key and
+// one warp reduction per bracket) instead of binary searches in shared memory, whose dependent loads
+// are what a lone lane spends its time on; the levels of the depth are counted one after the other,
+// then lane i finishes level i (the fp64 division of every level of the depth at the same time).
+// Positions past n hold the largest key, which no bracket reaches.  lvkey: the level keys in shared
+// memory, the brackets of this depth already in place.
+template <int KPT>
+__device__ __forceinline__ void bkt_depth_warp(const uint32_t (&r)[KPT], const uint32_t* keys, const double* pre,
+                                               uint32_t* lvkey, int s, int stride, int lane)
+{
+    int my_i0 = 0, my_i1 = 0, my_q = -1;
+    uint32_t my_kl = 0u, my_kr = 0u;
+    int idx = 0;
+    for (int q = stride; q < s - 1; q += 2 * stride, ++idx) {
+        const uint32_t kl = lvkey[q - stride], kr = lvkey[q + stride];
+        int i0 = 0, i1 = 0;
+        if (kr > kl) {
+            uint32_t below = 0u, upto = 0u;
+#pragma unroll
+            for (int e = 0; e < KPT; ++e) {
+                below += (r[e] < kl) ? 1u : 0u;
+                upto += (r[e] <= kr) ? 1u : 0u;
+            }
+            i0 = (int)__reduce_add_sync(0xffffffffu, below);
+            i1 = (int)__reduce_add_sync(0xffffffffu, upto);
+        }
+        if (lane == idx) { my_i0 = i0; my_i1 = i1; my_kl = kl; my_kr = kr; my_q = q; }
+    }
+    __syncwarp();
+    if (my_q >= 0) {
+        uint32_t res = my_kl;
+        if (my_kr > my_kl) {
+            const double Lv = (double)key_to_float(my_kl), Rv = (double)key_to_float(my_kr);
+            const int m = my_i1 - my_i0;
+            const double A = (pre[my_i1] - pre[my_i0]) - Lv * (double)m;
+            long long k = (long long)floor(A / (Rv - Lv));
+            if (k < 0) k = 0;
+            if (k > m - 1) k = m - 1;
+            res = keys[my_i1 - 1 - (int)k];
+        }
+        lvkey[my_q] = res;
+    }
+    __syncwarp();
 }
 
 // The same without prefix sums: called by every thread of the CTA, the segment's sum is a block sum.
@@ -290,12 +357,20 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
             const int P = KPT * blockDim.x;
             uint32_t r[KPT];
             int bad = 0;
+            // all loads first (positions past n read element 0 and are not used): written as one loop
+            // with the uses, the loads would be issued one global-memory latency after the other
+            float rawv[KPT];
+#pragma unroll
+            for (int e = 0; e < KPT; ++e) {
+                const int i = e * blockDim.x + threadIdx.x;
+                rawv[e] = __ldg(src + (i < n ? i : 0));
+            }
 #pragma unroll
             for (int e = 0; e < KPT; ++e) {
                 const int i = e * blockDim.x + threadIdx.x;
                 uint32_t key = 0xffffffffu;
                 if (i < n) {
-                    const float raw = __ldg(src + i);
+                    const float raw = rawv[e];
                     bad |= ((__float_as_uint(raw) & 0x7f800000u) == 0x7f800000u);
                     uint32_t bits = __float_as_uint(copysignf(fminf(fabsf(raw), tau), raw));
                     if (pbs) key = bits | 0x80000000u;
@@ -314,15 +389,19 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
             } else {
                 bkt_sort_regs<KPT>(r, keys, P);
                 __syncthreads();
+                static_assert(KPT % 4 == 0, "a thread's keys are stored as 128-bit words");
 #pragma unroll
-                for (int e = 0; e < KPT; ++e) keys[threadIdx.x * KPT + e] = r[e];
+                for (int e = 0; e < KPT; e += 4)
+                    *reinterpret_cast<uint4*>(keys + threadIdx.x * KPT + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
                 __syncthreads();
                 if (pre != nullptr) {
-                    // fp64 prefix sums of the sorted values: per-thread blocks, one scan over the threads
-                    const int per = (n + blockDim.x - 1) / blockDim.x;
-                    const int c0 = min((int)threadIdx.x * per, n), c1 = min(c0 + per, n);
+                    // fp64 prefix sums of the sorted values, from the registers that hold them (thread t
+                    // owns positions t * KPT ...): local sums, one scan over the threads, running sums out
+                    const int p0 = threadIdx.x * KPT;
                     double ls = 0.0;
-                    for (int i = c0; i < c1; ++i) ls += (double)key_to_float(keys[i]);
+#pragma unroll
+                    for (int e = 0; e < KPT; ++e)
+                        if (p0 + e < n) ls += (double)key_to_float(r[e]);
                     // exclusive scan of ls in thread order
                     double inc = ls;
 #pragma unroll
@@ -330,14 +409,18 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
                         const double nbv = __shfl_up_sync(0xffffffffu, inc, o);
                         if (lane >= o) inc = nbv + inc;
                     }
-                    __syncthreads();
-                    if (lane == 31) sh_d[warp] = inc;
-                    __syncthreads();
                     double wbase = 0.0;
-                    for (int w = 0; w < warp; ++w) wbase += sh_d[w];
+                    if (nwarps > 1) {
+                        __syncthreads();
+                        if (lane == 31) sh_d[warp] = inc;
+                        __syncthreads();
+                        for (int w = 0; w < warp; ++w) wbase += sh_d[w];
+                    }
                     double run = wbase + (inc - ls);
-                    for (int i = c0; i < c1; ++i) { pre[i] = run; run += (double)key_to_float(keys[i]); }
-                    if (c1 == n && c0 < n) pre[n] = run;
+#pragma unroll
+                    for (int e = 0; e < KPT; ++e)
+                        if (p0 + e < n) { pre[p0 + e] = run; run += (double)key_to_float(r[e]); }
+                    if (n > p0 && n <= p0 + KPT) pre[n] = run;
                     if (n == 0 && threadIdx.x == 0) pre[0] = 0.0;
                     __syncthreads();
                 }
@@ -347,7 +430,10 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
                     __syncthreads();
                     // Algorithm 1: a level after its two brackets, the levels of one depth side by side
                     for (int stride = (s - 1) >> 1; stride >= 1; stride >>= 1) {
-                        if (pre != nullptr) {
+                        if (pre != nullptr && nwarps == 1) {
+                            // one warp holds the bucket
+                            bkt_depth_warp<KPT>(r, keys, pre, sh_lvkey, s, stride, lane);
+                        } else if (pre != nullptr) {
                             const int q = threadIdx.x;
                             uint32_t res = 0u;
                             const bool mine = q < s - 1 && q >= stride && ((q - stride) % (2 * stride)) == 0;
@@ -451,10 +537,15 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
         }
         uint32_t* wsm = sh_words[warp];
         const int obit = (lane * 4 * BITS) & 31, oword = (lane * 4 * BITS) >> 5;
+        // (the next group's values are loaded before the current group is worked on)
+        const float4* src4 = reinterpret_cast<const float4*>(src) + lane;
+        float4 vnext = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (warp < nfull) vnext = __ldg(src4 + ((int64_t)warp << 5));
         for (int g = warp; g < ngroups; g += nwarps) {
             uint32_t bits4;
+            float4 v = vnext;
+            if (g + nwarps < nfull) vnext = __ldg(src4 + ((int64_t)(g + nwarps) << 5));
             if (g < nfull) {
-                float4 v = __ldg(reinterpret_cast<const float4*>(src + ((int64_t)g << 7)) + lane);
                 v.x = copysignf(fminf(fabsf(v.x), tau), v.x);  // clipping (tau = +Inf: none)
                 v.y = copysignf(fminf(fabsf(v.y), tau), v.y);
                 v.z = copysignf(fminf(fabsf(v.z), tau), v.z);
