@@ -279,15 +279,27 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
         __syncthreads();
         if (threadIdx.x == 0) { sh_flag = 0; sh_b0 = 0.f; }
         __syncthreads();
+        // The bucket's values, KPT per thread (element e * blockDim.x + threadIdx.x: coalesced), all loads
+        // issued before the first use; positions past n read element 0 and are not used.  Every later
+        // pass over the bucket but the quantizer's runs from these registers.
+        float rawv[KPT];
+#pragma unroll
+        for (int e = 0; e < KPT; ++e) {
+            const int i = e * blockDim.x + threadIdx.x;
+            rawv[e] = __ldg(src + (i < n ? i : 0));
+        }
         // clipping threshold of this bucket: c times the standard deviation about the mean (none: +Inf)
         float tau = __int_as_float(0x7f800000);
         if (A.clip_c > 0.f) {
             const double v0 = (double)__ldg(src);
             double s1 = 0.0, s2 = 0.0;
-            for (int i = threadIdx.x; i < n; i += blockDim.x) {
-                const double dv = (double)__ldg(src + i) - v0;
-                s1 += dv;
-                s2 += dv * dv;
+#pragma unroll
+            for (int e = 0; e < KPT; ++e) {
+                if (e * (int)blockDim.x + (int)threadIdx.x < n) {
+                    const double dv = (double)rawv[e] - v0;
+                    s1 += dv;
+                    s2 += dv * dv;
+                }
             }
             s1 = bkt_block_sum(s1, sh_d);
             s2 = bkt_block_sum(s2, sh_d);
@@ -300,10 +312,13 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
             // ---- BinGrad-b: b_0 = mean, b_{-1}, b_1 = conditional means, optional Lloyd updates
             double sum = 0.0;
             int bad = 0;
-            for (int i = threadIdx.x; i < n; i += blockDim.x) {
-                const float raw = __ldg(src + i);
-                bad |= ((__float_as_uint(raw) & 0x7f800000u) == 0x7f800000u);
-                sum += (double)copysignf(fminf(fabsf(raw), tau), raw);
+#pragma unroll
+            for (int e = 0; e < KPT; ++e) {
+                if (e * (int)blockDim.x + (int)threadIdx.x < n) {
+                    const float raw = rawv[e];
+                    bad |= ((__float_as_uint(raw) & 0x7f800000u) == 0x7f800000u);
+                    sum += (double)copysignf(fminf(fabsf(raw), tau), raw);
+                }
             }
             sum = bkt_block_sum(sum, sh_d);
             if (__syncthreads_or(bad)) stbits |= OGQ_ST_NONFINITE;
@@ -312,13 +327,16 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
             float l_lo = 0.f, l_hi = 0.f;
             for (int it = 0;; ++it) {
                 double s_lo = 0.0, s_hi = 0.0, c_lo = 0.0;
-                for (int i = threadIdx.x; i < n; i += blockDim.x) {
-                    const float raw = __ldg(src + i);
-                    const float v = copysignf(fminf(fabsf(raw), tau), raw);
-                    const bool below = v < b0;
-                    s_lo += below ? (double)v : 0.0;
-                    s_hi += below ? 0.0 : (double)v;
-                    c_lo += below ? 1.0 : 0.0;
+#pragma unroll
+                for (int e = 0; e < KPT; ++e) {
+                    if (e * (int)blockDim.x + (int)threadIdx.x < n) {
+                        const float raw = rawv[e];
+                        const float v = copysignf(fminf(fabsf(raw), tau), raw);
+                        const bool below = v < b0;
+                        s_lo += below ? (double)v : 0.0;
+                        s_hi += below ? 0.0 : (double)v;
+                        c_lo += below ? 1.0 : 0.0;
+                    }
                 }
                 s_lo = bkt_block_sum(s_lo, sh_d);
                 s_hi = bkt_block_sum(s_hi, sh_d);
@@ -357,14 +375,6 @@ k_bucket_encode(BktArgs A, const __grid_constant__ PhiloxKeys pk)
             const int P = KPT * blockDim.x;
             uint32_t r[KPT];
             int bad = 0;
-            // all loads first (positions past n read element 0 and are not used): written as one loop
-            // with the uses, the loads would be issued one global-memory latency after the other
-            float rawv[KPT];
-#pragma unroll
-            for (int e = 0; e < KPT; ++e) {
-                const int i = e * blockDim.x + threadIdx.x;
-                rawv[e] = __ldg(src + (i < n ? i : 0));
-            }
 #pragma unroll
             for (int e = 0; e < KPT; ++e) {
                 const int i = e * blockDim.x + threadIdx.x;
